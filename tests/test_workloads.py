@@ -1,0 +1,66 @@
+"""The seeded input generators: determinism, agreement of the two hash
+implementations, and the statistical shape the recipe promises."""
+import numpy as np
+import torch
+
+from workloads import (TINY, S7B, WORKLOADS, make_weights, markov_prompt, periodic_prompt,
+                       tensor_shapes)
+from workloads.rng import hash_at, hash_tensor, normal_tensor, MASK64
+
+
+def test_hash_python_and_torch_agree():
+    for seed, stream, start in [(0, 0, 0), (5, 3, 10), (2**40 + 7, 99, 12345)]:
+        h = hash_tensor(seed, stream, start, 64)
+        assert [x & MASK64 for x in h.tolist()] == [hash_at(seed, stream, start + i) for i in range(64)]
+
+
+def test_normal_moments_and_determinism():
+    a = normal_tensor(11, 4, 200_000, 0.02)
+    b = normal_tensor(11, 4, 200_000, 0.02, chunk=4096)
+    assert torch.equal(a, b)
+    assert abs(float(a.mean())) < 3e-4
+    assert abs(float(a.std()) - 0.02) < 3e-4
+    # tails exist (not a bounded approximation of a normal)
+    assert float(a.abs().max()) > 0.02 * 3.5
+    assert not torch.equal(a, normal_tensor(12, 4, 200_000, 0.02))
+
+
+def test_weight_set_names_and_streamed_bytes():
+    names = [n for n, _ in tensor_shapes(TINY)]
+    assert names[0] == "embed" and names[-1] == "lm_head" and len(names) == 1 + 9 * 2 + 2
+    w = make_weights(TINY, 0, False)
+    assert w["l1.w_down"].shape == (256, 688) and w["l0.attn_norm"].eq(1).all()
+    # bytes per verify step of the 7B shape quoted in the scope table: 13.214 GB + 524288 B/token
+    assert abs(S7B.streamed_params * 2 / 1e9 - 13.214) < 1e-3
+    assert S7B.kv_bytes_per_token == 524288
+    wb = make_weights(TINY, 0, True)
+    assert wb["l0.wq"].dtype == torch.bfloat16
+    assert torch.equal(wb["l0.wq"], w["l0.wq"].to(torch.bfloat16))
+
+
+def test_markov_prompt_shape():
+    wl = WORKLOADS["C3"]
+    p = markov_prompt(wl.prompt_len, wl.shape.vocab, 3, wl.prompt_seed, copy_spans=True)
+    q = markov_prompt(wl.prompt_len, wl.shape.vocab, 3, wl.prompt_seed, copy_spans=True)
+    assert p.dtype == np.int32 and p.shape == (1536,) and np.array_equal(p, q)
+    assert p.min() >= 0 and p.max() < wl.shape.vocab
+    # copied spans: a fair share of positions end an 8-gram already seen before
+    seen, rep = set(), 0
+    for i in range(8, len(p)):
+        g = tuple(p[i - 8:i])
+        rep += g in seen
+        seen.add(g)
+    assert 0.04 < rep / len(p) < 0.35
+    plain = markov_prompt(1536, wl.shape.vocab, 3, wl.prompt_seed, copy_spans=False)
+    seen, rep = set(), 0
+    for i in range(8, len(plain)):
+        g = tuple(plain[i - 8:i])
+        rep += g in seen
+        seen.add(g)
+    assert rep / len(plain) < 0.02
+
+
+def test_periodic_prompt():
+    p = periodic_prompt(40, 7, 100, 3)
+    assert len(set(p[:7].tolist())) == 7
+    assert all(p[i] == p[i % 7] for i in range(40))

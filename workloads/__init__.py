@@ -1,0 +1,10 @@
+"""Seeded synthetic inputs (weights, prompts) shared by the oracle's tests and
+the CUDA library's tests and benchmark.  Holds none of the method's arithmetic."""
+from .models import (ModelShape, Workload, WORKLOADS, TINY, S1B, S7B, S13B,
+                     tensor_shapes, make_weights, make_prompts)
+from .prompts import markov_prompt, periodic_prompt
+from . import rng
+
+__all__ = ["ModelShape", "Workload", "WORKLOADS", "TINY", "S1B", "S7B", "S13B",
+           "tensor_shapes", "make_weights", "make_prompts", "markov_prompt",
+           "periodic_prompt", "rng"]
