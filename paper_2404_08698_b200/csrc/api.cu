@@ -1,0 +1,586 @@
+// Handles, the verify / prefill / generate entry points and the measurement hooks.
+#include "internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+typedef __nv_bfloat16 bf16;
+
+long long g_launch_count = 0;
+static char g_last_error[256] = "";
+
+void anpd_note_cuda_error(cudaError_t e, const char* file, int line) {
+    std::snprintf(g_last_error, sizeof(g_last_error), "%s at %s:%d", cudaGetErrorString(e), file, line);
+    if (std::getenv("ANPD_VERBOSE")) std::fprintf(stderr, "[anpd] CUDA error: %s\n", g_last_error);
+    cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// profiler
+// ---------------------------------------------------------------------------------------------
+void Profiler::begin(cudaStream_t st, int c, double b) {
+    if (used * 2 + 2 > ev.size()) {
+        for (int i = 0; i < 2; ++i) { cudaEvent_t e; cudaEventCreate(&e); ev.push_back(e); }
+        cls.push_back(0); bytes.push_back(0);
+    }
+    cls[used] = c; bytes[used] = b;
+    cudaEventRecord(ev[used * 2], st);
+}
+void Profiler::end(cudaStream_t st) {
+    cudaEventRecord(ev[used * 2 + 1], st);
+    ++used;
+}
+void Profiler::drain() {
+    for (size_t i = 0; i < used; ++i) {
+        cudaEventSynchronize(ev[i * 2 + 1]);
+        float t = 0;
+        if (cudaEventElapsedTime(&t, ev[i * 2], ev[i * 2 + 1]) == cudaSuccess) {
+            ms[cls[i]] += t; n[cls[i]] += 1;
+            if (cls[i] == KC_GEMM) gemm_bytes += bytes[i];
+        }
+    }
+    used = 0;
+}
+void Profiler::clear() {
+    used = 0; gemm_bytes = 0;
+    for (int i = 0; i < KC_COUNT; ++i) { ms[i] = 0; n[i] = 0; }
+}
+Profiler::~Profiler() { for (cudaEvent_t e : ev) cudaEventDestroy(e); }
+
+namespace {
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = __float2bfloat16_rn(src[i]);
+}
+__global__ void set_int_kernel(int* p, int v) { *p = v; }
+__global__ void greedy_stage_kernel(SeqState* seqs) {
+    SeqState& s = seqs[blockIdx.x];
+    s.last_tok = s.next_tok;
+    s.draft_len = 0;
+}
+
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+uint16_t f32_to_bf16_host(float f) {
+    uint32_t u; std::memcpy(&u, &f, 4);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+// Copies one tensor into library memory as bf16 (matrices) or fp32 (norm gains).
+anpd_status upload(void* dst, const void* src, size_t n, bool as_bf16, bool src_bf16, bool on_device, cudaStream_t st,
+                   std::vector<uint16_t>& tmp, float* d_tmp, size_t d_tmp_elems) {
+    if (!as_bf16) {
+        CUDA_TRY(cudaMemcpyAsync(dst, src, n * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+        return ANPD_OK;
+    }
+    if (src_bf16) {
+        CUDA_TRY(cudaMemcpyAsync(dst, src, n * 2, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+        if (!on_device) CUDA_TRY(cudaStreamSynchronize(st));
+        return ANPD_OK;
+    }
+    if (on_device) {
+        LAUNCH(nullptr, st, KC_OTHER, 0, (f32_to_bf16_kernel<<<1024, 256, 0, st>>>((const float*)src, (bf16*)dst, n)));
+        CUDA_TRY(cudaGetLastError());
+        return ANPD_OK;
+    }
+    (void)d_tmp; (void)d_tmp_elems;
+    tmp.resize(n);
+    const float* f = (const float*)src;
+    for (size_t i = 0; i < n; ++i) tmp[i] = f32_to_bf16_host(f[i]);
+    CUDA_TRY(cudaMemcpyAsync(dst, tmp.data(), n * 2, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return ANPD_OK;
+}
+
+bool have_device() {
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || n == 0) { cudaGetLastError(); return false; }
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* anpd_status_string(anpd_status s) {
+    switch (s) {
+        case ANPD_OK: return "ok";
+        case ANPD_ERR_ARG: return "bad argument";
+        case ANPD_ERR_OOM: return "out of memory";
+        case ANPD_ERR_CAPACITY: return "capacity exceeded";
+        case ANPD_ERR_RANGE: return "value out of range";
+        case ANPD_ERR_CUDA: return g_last_error[0] ? g_last_error : "CUDA error";
+        case ANPD_ERR_STATE: return "call out of order";
+        default: return "unknown status";
+    }
+}
+
+long long anpd_launch_count(int reset) {
+    const long long v = g_launch_count;
+    if (reset) g_launch_count = 0;
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// model
+// ---------------------------------------------------------------------------------------------
+anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* weights, int weights_are_bf16,
+                              int weights_on_device, void* cuda_stream, anpd_model** out) {
+    if (!cfg || !weights || !out) return ANPD_ERR_ARG;
+    const anpd_model_config& c = *cfg;
+    if (c.n_layers < 1 || c.d_model < 8 || c.n_q_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 8 || c.vocab < 1) return ANPD_ERR_ARG;
+    if (c.head_dim != 64 && c.head_dim != 128) return ANPD_ERR_ARG;
+    if (c.n_q_heads % c.n_kv_heads != 0 || c.n_q_heads / c.n_kv_heads > 8) return ANPD_ERR_ARG;
+    if (c.d_model % 8 || c.d_ffn % 8 || c.vocab >= (1 << 24)) return ANPD_ERR_ARG;
+    if (!(c.rope_theta > 0.0f) || !(c.rms_eps >= 0.0f)) return ANPD_ERR_ARG;
+    const int n_tensors = 1 + 9 * c.n_layers + 2;
+    for (int i = 0; i < n_tensors; ++i) if (!weights[i]) return ANPD_ERR_ARG;
+    if (!have_device()) return ANPD_ERR_CUDA;
+
+    anpd_model* m = new (std::nothrow) anpd_model();
+    if (!m) return ANPD_ERR_OOM;
+    m->cfg = c;
+    m->stream = (cudaStream_t)cuda_stream;
+    m->dq = c.n_q_heads * c.head_dim;
+    m->dkv = c.n_kv_heads * c.head_dim;
+    m->nqkv = m->dq + 2 * m->dkv;
+    const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+    const size_t b_embed = up256(V * d * 2), b_qkv = up256((size_t)m->nqkv * d * 2), b_o = up256(d * m->dq * 2),
+                 b_gu = up256(2 * F * d * 2), b_d = up256(d * F * 2), b_norm = up256(d * 4);
+    m->slab_bytes = 2 * b_embed + b_norm + c.n_layers * (b_qkv + b_o + b_gu + b_d + 2 * b_norm);
+    if (cudaMalloc(&m->slab, m->slab_bytes) != cudaSuccess) { cudaGetLastError(); delete m; return ANPD_ERR_OOM; }
+    m->streamed_bytes = 2.0 * ((double)c.n_layers * ((double)m->nqkv * d + (double)d * m->dq + 3.0 * F * d) + (double)V * d);
+
+    char* p = (char*)m->slab;
+    std::vector<uint16_t> tmp;
+    const bool bf = weights_are_bf16 != 0, dev = weights_on_device != 0;
+    cudaStream_t st = m->stream;
+    anpd_status rc = ANPD_OK;
+    auto put = [&](const void* src, size_t n, bool as_bf16, size_t bytes) -> void* {
+        void* dst = p;
+        p += bytes;
+        if (rc == ANPD_OK) rc = upload(dst, src, n, as_bf16, bf, dev, st, tmp, nullptr, 0);
+        return dst;
+    };
+    int t = 0;
+    m->embed = (const bf16*)put(weights[t++], V * d, true, b_embed);
+    m->layers.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+        LayerW& w = m->layers[l];
+        w.attn_norm = (const float*)put(weights[t++], d, false, b_norm);
+        // q, k and v rows are stored back to back so that one GEMM produces all three
+        char* qkv = p;
+        put(weights[t++], (size_t)m->dq * d, true, (size_t)m->dq * d * 2);
+        put(weights[t++], (size_t)m->dkv * d, true, (size_t)m->dkv * d * 2);
+        put(weights[t++], (size_t)m->dkv * d, true, (size_t)m->dkv * d * 2);
+        p = qkv + b_qkv;
+        w.wqkv = (const bf16*)qkv;
+        w.wo = (const bf16*)put(weights[t++], d * m->dq, true, b_o);
+        w.ffn_norm = (const float*)put(weights[t++], d, false, b_norm);
+        char* gu = p;
+        put(weights[t++], F * d, true, F * d * 2);
+        put(weights[t++], F * d, true, F * d * 2);
+        p = gu + b_gu;
+        w.wgu = (const bf16*)gu;
+        w.wd = (const bf16*)put(weights[t++], d * F, true, b_d);
+    }
+    m->final_norm = (const float*)put(weights[t++], d, false, b_norm);
+    m->lm_head = (const bf16*)put(weights[t++], V * d, true, b_embed);
+    if (rc == ANPD_OK && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
+    if (rc != ANPD_OK) { cudaFree(m->slab); delete m; return rc; }
+    *out = m;
+    return ANPD_OK;
+}
+
+anpd_status anpd_model_destroy(anpd_model* m) {
+    if (!m) return ANPD_ERR_ARG;
+    cudaStreamSynchronize(m->stream);
+    cudaFree(m->slab);
+    delete m;
+    return ANPD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV cache + workspace
+// ---------------------------------------------------------------------------------------------
+anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shuffle_pages, anpd_kv** out) {
+    if (!cm || !out || max_len < ANPD_ROWS || batch < 1 || batch > 64) return ANPD_ERR_ARG;
+    anpd_model* m = const_cast<anpd_model*>(cm);
+    const anpd_model_config& c = m->cfg;
+    anpd_kv* kv = new (std::nothrow) anpd_kv();
+    if (!kv) return ANPD_ERR_OOM;
+    kv->m = m; kv->batch = batch;
+    kv->pages_per_seq = (max_len + KV_PAGE - 1) / KV_PAGE;
+    kv->max_len = kv->pages_per_seq * KV_PAGE;
+    kv->total_pages = kv->pages_per_seq * batch;
+    kv->staged = false;
+    kv->h_kv_len.assign(batch, 0);
+    Workspace& ws = kv->ws;
+    ws.r_max = std::max(PREFILL_ROWS, batch * ANPD_ROWS);
+    ws.n_max_out = std::max(std::max(m->nqkv, 2 * c.d_ffn), std::max(c.d_model, c.vocab));
+    ws.splits_max = 1;
+    ws.amax_blocks = (c.vocab + 1023) / 1024;
+    const size_t R = ws.r_max, d = c.d_model, F = c.d_ffn, V = c.vocab, hd = c.head_dim, half = hd / 2;
+    const size_t pool = (size_t)c.n_layers * kv->total_pages * c.n_kv_heads * KV_PAGE * hd * 2;
+    const size_t n_part = (size_t)R * c.n_q_heads * kv->pages_per_seq;
+    struct Item { void** ptr; size_t bytes; };
+    std::vector<Item> items = {
+        {(void**)&kv->kpool, pool}, {(void**)&kv->vpool, pool},
+        {(void**)&kv->page_table, (size_t)kv->total_pages * 4},
+        {(void**)&kv->rope_cos, (size_t)kv->max_len * half * 4}, {(void**)&kv->rope_sin, (size_t)kv->max_len * half * 4},
+        {(void**)&kv->seq, sizeof(SeqState) * (size_t)batch}, {(void**)&kv->d_prompt, (size_t)kv->max_len * 4},
+        {(void**)&kv->d_ctxs, sizeof(NgramDev) * (size_t)batch},
+        {(void**)&ws.row_tok, R * 4}, {(void**)&ws.row_pos, R * 4}, {(void**)&ws.row_seq, R * 4}, {(void**)&ws.row_ok, R * 4},
+        {(void**)&ws.x, R * d * 4}, {(void**)&ws.h_hi, R * d * 2}, {(void**)&ws.h_lo, R * d * 2},
+        {(void**)&ws.ao_hi, R * m->dq * 2}, {(void**)&ws.ao_lo, R * m->dq * 2},
+        {(void**)&ws.act_hi, R * F * 2}, {(void**)&ws.act_lo, R * F * 2},
+        {(void**)&ws.part, (size_t)ws.splits_max * R * ws.n_max_out * 4},
+        {(void**)&ws.q, R * m->dq * 4},
+        {(void**)&ws.attn_m, n_part * 4}, {(void**)&ws.attn_l, n_part * 4}, {(void**)&ws.attn_o, n_part * hd * 4},
+        {(void**)&ws.logits, R * V * 4},
+        {(void**)&ws.amax_val, R * ws.amax_blocks * 4}, {(void**)&ws.amax_idx, R * ws.amax_blocks * 4},
+    };
+    size_t total = 0;
+    for (const Item& it : items) total += up256(it.bytes);
+    kv->slab_bytes = total;
+    if (cudaMalloc(&kv->slab, total) != cudaSuccess) { cudaGetLastError(); delete kv; return ANPD_ERR_OOM; }
+    char* p = (char*)kv->slab;
+    for (const Item& it : items) { *it.ptr = p; p += up256(it.bytes); }
+    const size_t pinned_bytes = sizeof(SeqState) * (size_t)batch + 64 * sizeof(int) * (size_t)batch + 256;
+    if (cudaMallocHost((void**)&kv->h_seq, pinned_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(kv->slab); delete kv; return ANPD_ERR_OOM; }
+    kv->h_small = (int*)((char*)kv->h_seq + sizeof(SeqState) * (size_t)batch);
+
+    // page table: identity, or a fixed permutation of the physical pages
+    std::vector<int> pt(kv->total_pages);
+    for (int i = 0; i < kv->total_pages; ++i) pt[i] = i;
+    if (shuffle_pages) {
+        uint64_t s = 0x9E3779B97F4A7C15ull;
+        for (int i = kv->total_pages - 1; i > 0; --i) {
+            s = s * 6364136223846793005ull + 1442695040888963407ull;
+            std::swap(pt[i], pt[(int)((s >> 33) % (uint64_t)(i + 1))]);
+        }
+    }
+    // rotary tables in double, rounded once to fp32: angle = pos * theta^(-2i/hd)
+    std::vector<float> hc((size_t)kv->max_len * half), hs((size_t)kv->max_len * half);
+    for (size_t i = 0; i < half; ++i) {
+        const double inv = std::pow((double)c.rope_theta, -2.0 * (double)i / (double)hd);
+        for (int pos = 0; pos < kv->max_len; ++pos) {
+            hc[(size_t)pos * half + i] = (float)std::cos(pos * inv);
+            hs[(size_t)pos * half + i] = (float)std::sin(pos * inv);
+        }
+    }
+    cudaStream_t st = m->stream;
+    bool ok = cudaMemsetAsync(kv->slab, 0, total, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(kv->page_table, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(kv->rope_cos, hc.data(), hc.size() * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(kv->rope_sin, hs.data(), hs.size() * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    std::memset(kv->h_seq, 0, sizeof(SeqState) * (size_t)batch);
+    for (int b = 0; b < batch; ++b) { kv->h_seq[b].active = 1; kv->h_seq[b].stop_at = 0x7fffffff; }
+    ok = ok && cudaMemcpyAsync(kv->seq, kv->h_seq, sizeof(SeqState) * (size_t)batch, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) {
+        anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__);
+        cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv;
+        return ANPD_ERR_CUDA;
+    }
+    *out = kv;
+    return ANPD_OK;
+}
+
+anpd_status anpd_kv_destroy(anpd_kv* kv) {
+    if (!kv) return ANPD_ERR_ARG;
+    cudaStreamSynchronize(kv->m->stream);
+    cudaFreeHost(kv->h_seq);
+    cudaFree(kv->slab);
+    delete kv;
+    return ANPD_OK;
+}
+
+anpd_status anpd_kv_len(anpd_kv* kv, int seq, int* len) {
+    if (!kv || !len || seq < 0 || seq >= kv->batch) return ANPD_ERR_ARG;
+    *len = kv->h_kv_len[seq];
+    return ANPD_OK;
+}
+
+anpd_status anpd_kv_truncate(anpd_kv* kv, int seq, int len) {
+    if (!kv || seq < 0 || seq >= kv->batch || len < 0) return ANPD_ERR_ARG;
+    if (len > kv->h_kv_len[seq]) return ANPD_ERR_RANGE;
+    LAUNCH(&kv->m->prof, kv->m->stream, KC_OTHER, 0, (set_int_kernel<<<1, 1, 0, kv->m->stream>>>(&kv->seq[seq].kv_len, len)));
+    CUDA_TRY(cudaGetLastError());
+    kv->h_kv_len[seq] = len;
+    return ANPD_OK;
+}
+
+// Puts every sequence back to the empty state (device and host mirror).
+static anpd_status kv_reset(anpd_kv* kv, const int* stop_at) {
+    for (int b = 0; b < kv->batch; ++b) {
+        std::memset(&kv->h_seq[b], 0, sizeof(SeqState));
+        kv->h_seq[b].active = 1;
+        kv->h_seq[b].stop_at = stop_at ? stop_at[b] : 0x7fffffff;
+        kv->h_kv_len[b] = 0;
+    }
+    CUDA_TRY(cudaMemcpyAsync(kv->seq, kv->h_seq, sizeof(SeqState) * (size_t)kv->batch, cudaMemcpyHostToDevice, kv->m->stream));
+    CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
+    return ANPD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// prefill
+// ---------------------------------------------------------------------------------------------
+static anpd_status prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, const int32_t* prompt, int prompt_len,
+                                   const NgramDev* d_ctxs) {
+    CUDA_TRY(cudaMemcpyAsync(kv->d_prompt, prompt, sizeof(int) * (size_t)prompt_len, cudaMemcpyHostToDevice, m->stream));
+    for (int start = 0; start < prompt_len; start += PREFILL_ROWS) {
+        const int n = std::min(PREFILL_ROWS, prompt_len - start);
+        const int rows = (n + ANPD_ROWS - 1) / ANPD_ROWS * ANPD_ROWS;
+        const bool last = start + n >= prompt_len;
+        ANPD_TRY(plan_prefill_enqueue(m, kv, seq, start, prompt_len, rows));
+        ANPD_TRY(forward_enqueue(m, kv, rows, std::min(start + rows - 1, kv->max_len - 1), last, false));
+        if (last) ANPD_TRY(accept_enqueue(m, kv, ACCEPT_PREFILL, d_ctxs, seq, prompt_len - 1 - start, prompt_len));
+    }
+    return ANPD_OK;
+}
+
+static anpd_status read_seqs(anpd_kv* kv) {
+    CUDA_TRY(cudaMemcpyAsync(kv->h_seq, kv->seq, sizeof(SeqState) * (size_t)kv->batch, cudaMemcpyDeviceToHost, kv->m->stream));
+    CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
+    for (int b = 0; b < kv->batch; ++b) kv->h_kv_len[b] = kv->h_seq[b].kv_len;
+    return ANPD_OK;
+}
+
+static anpd_status seq_error_status(const SeqState& s) {
+    if (s.error == 0) return ANPD_OK;
+    if (s.error == 101) return ANPD_ERR_RANGE;
+    if (s.error == 102 || s.error == 103) return ANPD_ERR_CAPACITY;
+    return ANPD_ERR_CUDA;
+}
+
+anpd_status anpd_prefill(anpd_model* m, anpd_kv* kv, int seq, const int32_t* prompt, int prompt_len, int32_t* first_tok) {
+    if (!m || !kv || !prompt || !first_tok || kv->m != m || seq < 0 || seq >= kv->batch || prompt_len < 1) return ANPD_ERR_ARG;
+    if (kv->h_kv_len[seq] != 0) return ANPD_ERR_STATE;
+    if (prompt_len + ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
+    for (int i = 0; i < prompt_len; ++i) if (prompt[i] < 0 || prompt[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+    ANPD_TRY(prefill_enqueue(m, kv, seq, prompt, prompt_len, nullptr));
+    ANPD_TRY(read_seqs(kv));
+    ANPD_TRY(seq_error_status(kv->h_seq[seq]));
+    *first_tok = kv->h_seq[seq].next_tok;
+    return ANPD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// verify
+// ---------------------------------------------------------------------------------------------
+anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_tok, const int32_t* drafts, const int* draft_len) {
+    if (!m || !kv || kv->m != m || !last_tok || !draft_len) return ANPD_ERR_ARG;
+    const int B = kv->batch;
+    for (int b = 0; b < B; ++b) {
+        if (draft_len[b] < 0 || draft_len[b] > ANPD_K_MAX) return ANPD_ERR_RANGE;
+        if (draft_len[b] > 0 && !drafts) return ANPD_ERR_ARG;
+        if (last_tok[b] < 0 || last_tok[b] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+        for (int i = 0; i < draft_len[b]; ++i)
+            if (drafts[b * ANPD_K_MAX + i] < 0 || drafts[b * ANPD_K_MAX + i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+    }
+    // last_tok, draft_len and draft[] are adjacent in SeqState: one strided copy fills them
+    const int W = 2 + ANPD_K_MAX + 1;
+    CUDA_TRY(cudaStreamSynchronize(m->stream));          // the staging buffer may still be in use
+    int* stage = kv->h_small;
+    for (int b = 0; b < B; ++b) {
+        stage[b * W + 0] = last_tok[b];
+        stage[b * W + 1] = draft_len[b];
+        for (int i = 0; i <= ANPD_K_MAX; ++i) stage[b * W + 2 + i] = (i < draft_len[b]) ? drafts[b * ANPD_K_MAX + i] : 0;
+    }
+    CUDA_TRY(cudaMemcpy2DAsync(&kv->seq[0].last_tok, sizeof(SeqState), stage, W * sizeof(int), W * sizeof(int), B,
+                               cudaMemcpyHostToDevice, m->stream));
+    kv->staged = true;
+    return ANPD_OK;
+}
+
+static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs) {
+    int max_pos = 0;
+    for (int b = 0; b < kv->batch; ++b) {
+        if (kv->h_kv_len[b] + ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
+        max_pos = std::max(max_pos, kv->h_kv_len[b] + ANPD_ROWS - 1);
+    }
+    ANPD_TRY(plan_decode_enqueue(m, kv));
+    ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
+    ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
+    return ANPD_OK;
+}
+
+anpd_status anpd_verify_enqueue(anpd_model* m, anpd_kv* kv) {
+    if (!m || !kv || kv->m != m) return ANPD_ERR_ARG;
+    if (!kv->staged) return ANPD_ERR_STATE;
+    return verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, nullptr);
+}
+
+anpd_status anpd_verify_result(anpd_model* m, anpd_kv* kv, int* accepted_len, int32_t* next_tok) {
+    if (!m || !kv || kv->m != m || !accepted_len || !next_tok) return ANPD_ERR_ARG;
+    ANPD_TRY(read_seqs(kv));
+    for (int b = 0; b < kv->batch; ++b) ANPD_TRY(seq_error_status(kv->h_seq[b]));
+    for (int b = 0; b < kv->batch; ++b) { accepted_len[b] = kv->h_seq[b].accepted_len; next_tok[b] = kv->h_seq[b].next_tok; }
+    return ANPD_OK;
+}
+
+anpd_status anpd_verify_batch(anpd_model* m, anpd_kv* kv, const int32_t* last_tok, const int32_t* drafts,
+                              const int* draft_len, int* accepted_len, int32_t* next_tok) {
+    if (!accepted_len || !next_tok) return ANPD_ERR_ARG;
+    ANPD_TRY(anpd_verify_stage(m, kv, last_tok, drafts, draft_len));
+    ANPD_TRY(anpd_verify_enqueue(m, kv));
+    return anpd_verify_result(m, kv, accepted_len, next_tok);
+}
+
+anpd_status anpd_verify(anpd_model* m, anpd_kv* kv, int32_t last_tok, const int32_t* draft, int draft_len,
+                        int* accepted_len, int32_t* next_tok) {
+    if (!kv || kv->batch != 1) return ANPD_ERR_ARG;
+    int32_t padded[ANPD_K_MAX] = {0};
+    if (draft_len < 0 || draft_len > ANPD_K_MAX) return ANPD_ERR_RANGE;
+    if (draft_len > 0 && !draft) return ANPD_ERR_ARG;
+    for (int i = 0; i < draft_len; ++i) padded[i] = draft[i];
+    return anpd_verify_batch(m, kv, &last_tok, padded, &draft_len, accepted_len, next_tok);
+}
+
+anpd_status anpd_verify_logits(anpd_model* m, anpd_kv* kv, int32_t last_tok, const int32_t* draft, int draft_len,
+                               float* logits_host) {
+    if (!kv || kv->batch != 1 || !logits_host) return ANPD_ERR_ARG;
+    int32_t padded[ANPD_K_MAX] = {0};
+    if (draft_len < 0 || draft_len > ANPD_K_MAX) return ANPD_ERR_RANGE;
+    if (draft_len > 0 && !draft) return ANPD_ERR_ARG;
+    for (int i = 0; i < draft_len; ++i) padded[i] = draft[i];
+    ANPD_TRY(anpd_verify_stage(m, kv, &last_tok, padded, &draft_len));
+    ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_PEEK, true, nullptr));
+    CUDA_TRY(cudaMemcpyAsync(logits_host, kv->ws.logits, sizeof(float) * (size_t)(draft_len + 1) * m->cfg.vocab,
+                             cudaMemcpyDeviceToHost, m->stream));
+    ANPD_TRY(read_seqs(kv));
+    return seq_error_status(kv->h_seq[0]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Algorithm 1
+// ---------------------------------------------------------------------------------------------
+anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* ctxs, const int32_t* prompts,
+                                int prompt_len, int max_new, int K, int32_t* out, anpd_stats* stats) {
+    if (!m || !kv || kv->m != m || !ctxs || !prompts || !out || prompt_len < 1 || max_new < 1) return ANPD_ERR_ARG;
+    if (K < 0 || K > ANPD_K_MAX) return ANPD_ERR_RANGE;
+    const int B = kv->batch;
+    cudaStream_t st = m->stream;
+    for (int b = 0; b < B; ++b) {
+        if (!ctxs[b] || ctxs[b]->stream != st) return ANPD_ERR_ARG;
+        if (prompt_len + max_new + ANPD_ROWS > ctxs[b]->h.max_ctx) return ANPD_ERR_CAPACITY;
+    }
+    if (prompt_len + max_new + 2 * ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
+    for (size_t i = 0; i < (size_t)B * prompt_len; ++i) if (prompts[i] < 0 || prompts[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+
+    std::vector<int> stop(B, prompt_len + max_new);
+    ANPD_TRY(kv_reset(kv, stop.data()));
+    std::vector<NgramDev> hd(B);
+    for (int b = 0; b < B; ++b) {
+        ANPD_TRY(anpd_ngram_reset(ctxs[b]));
+        hd[b] = ctxs[b]->h;
+    }
+    CUDA_TRY(cudaMemcpyAsync(kv->d_ctxs, hd.data(), sizeof(NgramDev) * (size_t)B, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+
+    cudaEvent_t e0, e1, e2;
+    CUDA_TRY(cudaEventCreate(&e0)); CUDA_TRY(cudaEventCreate(&e1)); CUDA_TRY(cudaEventCreate(&e2));
+    anpd_status rc = ANPD_OK;
+    auto body = [&]() -> anpd_status {
+        CUDA_TRY(cudaEventRecord(e0, st));
+        // Initialize: the prompt's statistics (skipped for plain greedy, which never queries them)
+        for (int b = 0; b < B; ++b) {
+            anpd_ngram* c = ctxs[b];
+            CUDA_TRY(cudaMemcpyAsync(c->h.tokens, prompts + (size_t)b * prompt_len, sizeof(int) * (size_t)prompt_len,
+                                     cudaMemcpyHostToDevice, st));
+            kv->h_small[2 * b] = prompt_len; kv->h_small[2 * b + 1] = (K > 0) ? prompt_len : 0;
+            CUDA_TRY(cudaMemcpyAsync(c->h.state, kv->h_small + 2 * b, 2 * sizeof(int), cudaMemcpyHostToDevice, st));
+            if (K > 0) ANPD_TRY(ngram_enqueue_bulk(c, 0, prompt_len, &m->prof));
+        }
+        // LLM(prompt): the first token lands in the context as its first uncounted token
+        for (int b = 0; b < B; ++b) ANPD_TRY(prefill_enqueue(m, kv, b, prompts + (size_t)b * prompt_len, prompt_len, kv->d_ctxs));
+        CUDA_TRY(cudaEventRecord(e1, st));
+        ANPD_TRY(read_seqs(kv));
+        for (int b = 0; b < B; ++b) ANPD_TRY(seq_error_status(kv->h_seq[b]));
+        bool any_active = true;
+        while (any_active) {
+            if (K > 0) ANPD_TRY(ngram_enqueue_step(kv->d_ctxs, kv->seq, B, K, st, &m->prof));
+            else { LAUNCH(&m->prof, st, KC_OTHER, 0, (greedy_stage_kernel<<<B, 1, 0, st>>>(kv->seq))); }
+            ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs));
+            ANPD_TRY(read_seqs(kv));
+            any_active = false;
+            for (int b = 0; b < B; ++b) {
+                ANPD_TRY(seq_error_status(kv->h_seq[b]));
+                any_active = any_active || kv->h_seq[b].active;
+            }
+        }
+        CUDA_TRY(cudaEventRecord(e2, st));
+        CUDA_TRY(cudaEventSynchronize(e2));
+        return ANPD_OK;
+    };
+    rc = body();
+    if (rc == ANPD_OK) {
+        float ms_p = 0, ms_d = 0;
+        cudaEventElapsedTime(&ms_p, e0, e1);
+        cudaEventElapsedTime(&ms_d, e1, e2);
+        for (int b = 0; b < B && rc == ANPD_OK; ++b) {
+            if (cudaMemcpy(out + (size_t)b * max_new, ctxs[b]->h.tokens + prompt_len, sizeof(int) * (size_t)max_new,
+                           cudaMemcpyDeviceToHost) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; break; }
+            int nst[2] = {0, 0};
+            if (cudaMemcpy(nst, ctxs[b]->h.state, 2 * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = ANPD_ERR_CUDA; break; }
+            const int nt = nst[0];
+            ctxs[b]->n_tokens = nt;
+            ctxs[b]->n_folded = (K > 0) ? nst[1] : 0;
+            if (stats) {
+                const SeqState& s = kv->h_seq[b];
+                anpd_stats& o = stats[b];
+                o.steps = s.steps; o.drafted = s.drafted; o.accepted = s.accepted; o.generated = nt - prompt_len;
+                for (int i = 0; i < 8; ++i) o.hist_accepted[i] = s.hist[i];
+                o.ms_prefill = ms_p; o.ms_decode = ms_d;
+                const double mean_kv = prompt_len + 0.5 * (nt - prompt_len);
+                const anpd_model_config& c = m->cfg;
+                o.bytes_per_step = m->streamed_bytes + B * mean_kv * (2.0 * c.n_layers * c.n_kv_heads * c.head_dim * 2.0);
+            }
+        }
+    }
+    cudaEventDestroy(e0); cudaEventDestroy(e1); cudaEventDestroy(e2);
+    return rc;
+}
+
+anpd_status anpd_generate(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const int32_t* prompt, int prompt_len,
+                          int max_new, int K, int32_t* out, int* n_out, anpd_stats* stats) {
+    if (!kv || kv->batch != 1 || !n_out) return ANPD_ERR_ARG;
+    anpd_ngram* arr[1] = {ctx};
+    ANPD_TRY(anpd_generate_batch(m, kv, arr, prompt, prompt_len, max_new, K, out, stats));
+    *n_out = max_new;
+    return ANPD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// measurement
+// ---------------------------------------------------------------------------------------------
+anpd_status anpd_profile_enable(anpd_model* m, int on) {
+    if (!m) return ANPD_ERR_ARG;
+    CUDA_TRY(cudaStreamSynchronize(m->stream));
+    m->prof.drain();
+    m->prof.on = on != 0;
+    return ANPD_OK;
+}
+
+anpd_status anpd_profile_read(anpd_model* m, anpd_profile* out, int reset) {
+    if (!m || !out) return ANPD_ERR_ARG;
+    CUDA_TRY(cudaStreamSynchronize(m->stream));
+    m->prof.drain();
+    out->ms_gemm = m->prof.ms[KC_GEMM]; out->n_gemm = m->prof.n[KC_GEMM];
+    out->ms_attn = m->prof.ms[KC_ATTN]; out->n_attn = m->prof.n[KC_ATTN];
+    out->ms_other = m->prof.ms[KC_OTHER]; out->n_other = m->prof.n[KC_OTHER];
+    out->ms_ngram = m->prof.ms[KC_NGRAM]; out->n_ngram = m->prof.n[KC_NGRAM];
+    out->gemm_bytes = m->prof.gemm_bytes;
+    if (reset) m->prof.clear();
+    return ANPD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,201 @@
+// Internal declarations shared by the library's translation units (not part of the boundary).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <vector>
+
+#include "anpd.h"
+
+// ---------------------------------------------------------------------------------------------
+// error handling
+// ---------------------------------------------------------------------------------------------
+void anpd_note_cuda_error(cudaError_t e, const char* file, int line);
+
+#define CUDA_TRY(expr)                                            \
+    do {                                                          \
+        cudaError_t e__ = (expr);                                 \
+        if (e__ != cudaSuccess) {                                 \
+            anpd_note_cuda_error(e__, __FILE__, __LINE__);        \
+            return ANPD_ERR_CUDA;                                 \
+        }                                                         \
+    } while (0)
+
+#define ANPD_TRY(expr)                       \
+    do {                                     \
+        anpd_status s__ = (expr);            \
+        if (s__ != ANPD_OK) return s__;      \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// launch accounting + optional per-class timing
+// ---------------------------------------------------------------------------------------------
+enum KernelClass { KC_GEMM = 0, KC_ATTN = 1, KC_OTHER = 2, KC_NGRAM = 3, KC_COUNT = 4 };
+
+struct Profiler {
+    bool on = false;
+    std::vector<cudaEvent_t> ev;      // pairs
+    std::vector<int> cls;             // class per pair
+    std::vector<double> bytes;        // bytes per pair (GEMM weight bytes)
+    size_t used = 0;                  // pairs in use
+    double ms[KC_COUNT] = {0, 0, 0, 0};
+    int n[KC_COUNT] = {0, 0, 0, 0};
+    double gemm_bytes = 0;
+    void begin(cudaStream_t st, int c, double b);
+    void end(cudaStream_t st);
+    void drain();                     // synchronises the events and folds them into ms/n
+    void clear();
+    ~Profiler();
+};
+
+extern long long g_launch_count;
+
+// Wraps one kernel launch: counts it and, when profiling, brackets it with events.
+#define LAUNCH(prof, stream, kclass, wbytes, ...)                      \
+    do {                                                               \
+        Profiler* p__ = (prof);                                        \
+        if (p__ && p__->on) p__->begin((stream), (kclass), (wbytes));  \
+        __VA_ARGS__;                                                   \
+        ++g_launch_count;                                              \
+        if (p__ && p__->on) p__->end((stream));                        \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// per-sequence step state (device)
+// ---------------------------------------------------------------------------------------------
+struct SeqState {
+    int kv_len;                    // P: positions held by the cache
+    int last_tok;                  // confirmed token fed as row 0
+    int draft_len;                 // k <= K
+    int draft[ANPD_K_MAX + 1];
+    int accepted_len;              // a
+    int next_tok;                  // the model's token after the last accepted draft
+    int pred[ANPD_ROWS];           // argmax per row
+    int steps, drafted, accepted;  // counters of the decoding loop
+    int hist[8];
+    int active;                    // 0: the sequence idles (finished or out of room)
+    int stop_at;                   // the loop retires the sequence once its context holds this many tokens
+    int error;                     // sticky device-side error code
+};
+
+// ---------------------------------------------------------------------------------------------
+// n-gram tables (device)
+// ---------------------------------------------------------------------------------------------
+// Both tables of a level identify a key by a position: ref = t + 1 where t is a position of the
+// committed sequence at which the n-gram x[t-n+1..t] occurred (0 = empty slot).  The key's
+// tokens are read from the token buffer, which never changes below n_tokens.
+struct GramSlot {      // one record per distinct n-gram
+    int ref;
+    int count;         // occurrences
+    int last;          // last position t
+    int pad;
+};
+struct PrefSlot {      // one record per distinct (n-1)-gram context
+    int ref;
+    int pad;
+    unsigned long long best;   // packed (count | last_pos | successor), larger is better
+};
+
+struct NgramDev {
+    int* tokens;       // [max_ctx]
+    int* state;        // [0] n_tokens, [1] first position not yet folded into the tables, [2] error
+    GramSlot* gram[ANPD_N_MAX + 1];   // indexed by n
+    PrefSlot* pref[ANPD_N_MAX + 1];
+    int n_min, n_max, max_ctx, cap, policy;
+};
+
+struct anpd_ngram {
+    NgramDev h;            // host copy of the descriptor (device pointers inside)
+    NgramDev* d;           // device copy, for kernels that take an array of descriptors
+    cudaStream_t stream;
+    int n_tokens;          // host mirror, valid whenever no asynchronous loop is running
+    int n_folded;          // host mirror of state[1]: tokens below it are in the tables
+    int* pinned;           // small pinned staging buffer
+    void* slab;            // all tables, one allocation
+    size_t slab_bytes;
+};
+
+anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof);
+// One fused launch for `batch` sequences: folds tokens [state[1], state[0]) of each, then drafts
+// K tokens into seq[b] (draft, draft_len, last_tok).
+anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batch, int K,
+                               cudaStream_t st, Profiler* prof);
+
+// ---------------------------------------------------------------------------------------------
+// model, KV cache and workspace
+// ---------------------------------------------------------------------------------------------
+constexpr int KV_PAGE = 128;          // positions per KV page (= key chunk of one attention block)
+constexpr int PREFILL_ROWS = 64;      // rows per prefill pass
+
+struct LayerW {
+    const __nv_bfloat16* wqkv;        // [(Hq + 2 Hkv) * hd, d]  (q rows, then k rows, then v rows)
+    const __nv_bfloat16* wo;          // [d, Hq * hd]
+    const __nv_bfloat16* wgu;         // [2 F, d]  (gate rows, then up rows)
+    const __nv_bfloat16* wd;          // [d, F]
+    const float* attn_norm;           // [d]
+    const float* ffn_norm;            // [d]
+};
+
+struct anpd_model {
+    anpd_model_config cfg;
+    cudaStream_t stream;
+    int dq, dkv, nqkv;
+    const __nv_bfloat16* embed;       // [V, d]
+    const __nv_bfloat16* lm_head;     // [V, d]
+    const float* final_norm;          // [d]
+    std::vector<LayerW> layers;
+    void* slab;
+    size_t slab_bytes;
+    double streamed_bytes;            // weight bytes one forward reads
+    Profiler prof;
+};
+
+struct Workspace {
+    int r_max;                        // rows any forward may use
+    int n_max_out;                    // widest GEMM output (max of nqkv, 2F, d, V)
+    int splits_max;
+    int* row_tok; int* row_pos; int* row_seq; int* row_ok;    // [r_max]
+    float* x;                         // [r_max, d] residual stream
+    __nv_bfloat16 *h_hi, *h_lo;       // [r_max, d]   normalised input of QKV / gate-up / LM head
+    __nv_bfloat16 *ao_hi, *ao_lo;     // [r_max, dq]  attention output, input of the O projection
+    __nv_bfloat16 *act_hi, *act_lo;   // [r_max, F]   SwiGLU output, input of the down projection
+    float* part;                      // [splits_max, r_max, n_max_out] GEMM partial sums
+    float* q;                         // [r_max, dq]
+    float *attn_m, *attn_l, *attn_o;  // per (row, q head, key chunk): max, sum, weighted values
+    float* logits;                    // [r_max, V]
+    float* amax_val; int* amax_idx;   // [r_max, amax_blocks]
+    int amax_blocks;
+};
+
+struct anpd_kv {
+    anpd_model* m;
+    int batch, max_len, pages_per_seq, total_pages;
+    __nv_bfloat16 *kpool, *vpool;     // [L][total_pages][Hkv][KV_PAGE][hd]
+    int* page_table;                  // device [batch][pages_per_seq]
+    float *rope_cos, *rope_sin;       // [max_len][hd/2]
+    SeqState* seq;                    // device [batch]
+    SeqState* h_seq;                  // pinned host staging [batch]
+    int* d_prompt;                    // device [max_len]
+    NgramDev* d_ctxs;                 // device [batch]: descriptors of the sequences' n-gram contexts
+    int* h_small;                     // pinned, a few ints
+    std::vector<int> h_kv_len;        // host mirror of the sequences' lengths
+    Workspace ws;
+    void* slab;
+    size_t slab_bytes;
+    bool staged;
+};
+
+// Forward over `rows` rows (a multiple of 8; 8 consecutive rows always belong to one sequence and
+// hold consecutive positions).  The row plan (ws.row_*) must have been written on the stream.
+// max_pos: an upper bound of the largest position any row holds (sizes the attention grid).
+// head: also run the LM head and the per-block argmax (false for all but the last prefill pass).
+anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits);
+
+enum AcceptMode { ACCEPT_COMMIT = 0, ACCEPT_PEEK = 1, ACCEPT_PREFILL = 2 };
+anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv);
+anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start, int prompt_len, int rows);
+// mode COMMIT/PEEK: one block per sequence over its 8 rows.  PREFILL: `last_row` of sequence
+// `seq` gives the first generated token, kv_len becomes prompt_len.  d_ctxs may be null; otherwise
+// accepted tokens and the next token are appended to the sequences' token buffers.
+anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len);

@@ -1,0 +1,207 @@
+"""The CUDA verify forward against the oracle decoder: logits within 2e-2 (bf16 operands and
+bf16 KV cache on the GPU, fp64 on the CPU), decisions equal wherever the oracle's top-2 margin
+exceeds 5e-2, and bit-identical results regardless of row count or page order."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import as_bf16_values, gpu_model, require_gpu, top2_margin
+from oracle.anpd import accept_length, argmax_lowest
+from oracle.decoder import Decoder
+from workloads import WORKLOADS, ModelShape, make_prompts, make_weights, markov_prompt
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = 2e-2      # max-abs, GPU bf16 path vs CPU oracle
+MARGIN = 5e-2         # decisions are compared only where the oracle's top-2 margin exceeds this
+
+
+@pytest.fixture(scope="module")
+def A():
+    require_gpu()
+    from paper_2404_08698_b200 import binding
+    return binding
+
+
+class Rig:
+    def __init__(self, A, shape, seed=0, std=0.02, jitter=0.0, max_len=512, shuffle=False, bf16=False):
+        self.A, self.shape = A, shape
+        self.w = make_weights(shape, seed, bf16, std=std, norm_gain_jitter=jitter)
+        self.m = gpu_model(A, shape, self.w)
+        self.kv = A.anpd_kv_create(self.m, max_len, 1, shuffle)
+        self.dec = Decoder(shape, {k: v.float() if v.dim() == 2 else v for k, v in self.w.items()}, torch.float64)
+        self.dec_bf16 = Decoder(shape, as_bf16_values(self.w), torch.float64)
+
+    def close(self):
+        self.A.anpd_kv_destroy(self.kv)
+        self.A.anpd_model_destroy(self.m)
+
+
+@pytest.fixture(scope="module")
+def c1(A):
+    r = Rig(A, WORKLOADS["C1"].shape)
+    yield r
+    r.close()
+
+
+def test_c1_logits_parity_after_prefill(A, c1):
+    wl = WORKLOADS["C1"]
+    prompt = make_prompts(wl)[0].tolist()
+    A.anpd_kv_truncate(c1.kv, 0, 0)
+    first = A.anpd_prefill(c1.m, c1.kv, prompt)
+    assert A.anpd_kv_len(c1.kv) == len(prompt)
+    cache = c1.dec.new_cache()
+    lp = c1.dec.forward(prompt, cache)
+    if top2_margin(lp[-1]) > MARGIN:
+        assert first == argmax_lowest(lp[-1])
+    # a verify step with a 7-token draft: all 8 rows against the oracle's logits
+    draft = [int(t) for t in prompt[3:10]]
+    got = A.anpd_verify_logits(c1.m, c1.kv, first, draft, wl.shape.vocab)
+    assert A.anpd_kv_len(c1.kv) == len(prompt)                     # the hook commits nothing
+    want = c1.dec.forward([first] + draft, cache)
+    err = float((torch.from_numpy(got).double() - want).abs().max())
+    assert err <= LOGIT_TOL, err
+    # against the oracle on the bf16-rounded weight values only activation/KV rounding is left
+    cb = c1.dec_bf16.new_cache()
+    c1.dec_bf16.forward(prompt, cb)
+    want_b = c1.dec_bf16.forward([first] + draft, cb)
+    err_b = float((torch.from_numpy(got).double() - want_b).abs().max())
+    assert err_b <= 5e-3, err_b
+
+
+def test_verify_decisions_match_oracle(A, c1):
+    wl = WORKLOADS["C1"]
+    prompt = make_prompts(wl)[0].tolist()
+    A.anpd_kv_truncate(c1.kv, 0, 0)
+    last = A.anpd_prefill(c1.m, c1.kv, prompt)
+    cache = c1.dec_bf16.new_cache()
+    c1.dec_bf16.forward(prompt, cache)
+    rng = np.random.default_rng(0)
+    checked = 0
+    for step in range(12):
+        # build a draft that follows the oracle's own predictions for a random number of tokens
+        P = cache.length
+        k = int(rng.integers(0, 8))
+        good = int(rng.integers(0, k + 1))
+        draft, rows = [], [last]
+        for i in range(k):
+            lg = c1.dec_bf16.forward([rows[-1]], cache)
+            t = argmax_lowest(lg[-1])
+            if i >= good:
+                t = (t + 1 + int(rng.integers(0, 5))) % wl.shape.vocab
+            draft.append(t)
+            rows.append(t)
+        cache.truncate(P)
+        logits = c1.dec_bf16.forward([last] + draft, cache)
+        preds = [argmax_lowest(logits[r]) for r in range(k + 1)]
+        a_want = accept_length(draft, preds)
+        safe = all(top2_margin(logits[r]) > MARGIN for r in range(a_want + 1))
+        a, nxt = A.anpd_verify(c1.m, c1.kv, last, draft)
+        if not safe:
+            break
+        assert (a, nxt) == (a_want, preds[a_want]), (step, draft, preds)
+        assert a >= min(good, k)
+        assert A.anpd_kv_len(c1.kv) == P + a + 1
+        cache.truncate(P + a + 1)
+        last = nxt
+        checked += 1
+    assert checked >= 3
+
+
+def test_rows_are_independent_of_row_count_and_drafts(A, c1):
+    wl = WORKLOADS["C1"]
+    prompt = make_prompts(wl)[0].tolist()[:100]
+    A.anpd_kv_truncate(c1.kv, 0, 0)
+    first = A.anpd_prefill(c1.m, c1.kv, prompt)
+    draft = prompt[10:17]
+    full = A.anpd_verify_logits(c1.m, c1.kv, first, draft, wl.shape.vocab)          # 8 real rows
+    one = A.anpd_verify_logits(c1.m, c1.kv, first, [], wl.shape.vocab)              # 1 real row
+    assert np.array_equal(full[0], one[0])
+    part = A.anpd_verify_logits(c1.m, c1.kv, first, draft[:3], wl.shape.vocab)
+    assert np.array_equal(full[:4], part)
+    # row r of the wide step == row 0 of a one-row step taken after committing r tokens
+    seq = [first] + draft
+    for r in range(1, 6):
+        # commit exactly one more token: a step whose (empty) draft accepts nothing
+        A.anpd_verify(c1.m, c1.kv, seq[r - 1], [])
+        assert A.anpd_kv_len(c1.kv) == len(prompt) + r
+        single = A.anpd_verify_logits(c1.m, c1.kv, seq[r], [], wl.shape.vocab)
+        assert np.array_equal(single[0], full[r]), r
+    # roll back and redo: same bits again
+    A.anpd_kv_truncate(c1.kv, 0, len(prompt))
+    again = A.anpd_verify_logits(c1.m, c1.kv, first, draft, wl.shape.vocab)
+    assert np.array_equal(again, full)
+
+
+def test_page_order_does_not_matter(A):
+    shape = WORKLOADS["C1"].shape
+    prompt = markov_prompt(300, shape.vocab, 2, 77).tolist()          # three pages, ragged tail
+    outs = []
+    for shuffle in (False, True):
+        r = Rig(A, shape, max_len=512, shuffle=shuffle)
+        try:
+            first = A.anpd_prefill(r.m, r.kv, prompt)
+            outs.append((first, A.anpd_verify_logits(r.m, r.kv, first, prompt[5:12], shape.vocab)))
+        finally:
+            r.close()
+    assert outs[0][0] == outs[1][0] and np.array_equal(outs[0][1], outs[1][1])
+
+
+@pytest.mark.parametrize("shape,plen", [
+    (ModelShape(2, 128, 8, 2, 64, 200, 512), 150),      # grouped-query, 4 q heads per kv head, hd 64
+    (ModelShape(1, 256, 2, 2, 128, 264, 300), 131),     # hd 128, ragged vocab / ffn
+    (ModelShape(2, 128, 8, 1, 64, 136, 1030), 9),       # 8 q heads on one kv head, prompt shorter than a pass
+])
+def test_other_shapes_logits_parity(A, shape, plen):
+    r = Rig(A, shape, seed=11, std=0.05, jitter=0.1, max_len=256)
+    try:
+        prompt = markov_prompt(plen, shape.vocab, 2, 5).tolist()
+        first = A.anpd_prefill(r.m, r.kv, prompt)
+        cache = r.dec_bf16.new_cache()
+        lp = r.dec_bf16.forward(prompt, cache)
+        if top2_margin(lp[-1]) > MARGIN:
+            assert first == argmax_lowest(lp[-1])
+        draft = prompt[1:6]
+        got = A.anpd_verify_logits(r.m, r.kv, first, draft, shape.vocab)
+        want = r.dec_bf16.forward([first] + draft, cache)
+        err = float((torch.from_numpy(got).double() - want).abs().max())
+        assert err <= LOGIT_TOL, err
+    finally:
+        r.close()
+
+
+def test_bf16_weight_input_equals_fp32_input_rounded(A):
+    shape = ModelShape(1, 64, 1, 1, 64, 64, 128)
+    w32 = make_weights(shape, 4, False, std=0.1)
+    w16 = {k: (v.to(torch.bfloat16) if v.dim() == 2 else v) for k, v in w32.items()}
+    outs = []
+    for w in (w32, w16, {k: v.cuda() for k, v in w16.items()}):
+        m = gpu_model(A, shape, w)
+        kv = A.anpd_kv_create(m, 64)
+        try:
+            first = A.anpd_prefill(m, kv, [1, 2, 3, 4, 5])
+            outs.append(A.anpd_verify_logits(m, kv, first, [7, 8], shape.vocab))
+        finally:
+            A.anpd_kv_destroy(kv)
+            A.anpd_model_destroy(m)
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[1], outs[2])
+
+
+def test_verify_error_paths(A, c1):
+    A.anpd_kv_truncate(c1.kv, 0, 0)
+    with pytest.raises(A.AnpdError) as e:
+        A.anpd_verify(c1.m, c1.kv, 4096, [])                           # token id == vocab
+    assert e.value.status == A.ERR_RANGE
+    with pytest.raises(A.AnpdError) as e:
+        A.anpd_verify(c1.m, c1.kv, 1, list(range(8)))                  # K > 7
+    assert e.value.status == A.ERR_RANGE
+    A.anpd_prefill(c1.m, c1.kv, [1, 2, 3])
+    with pytest.raises(A.AnpdError) as e:
+        A.anpd_prefill(c1.m, c1.kv, [1, 2, 3])                         # cache not empty
+    assert e.value.status == A.ERR_STATE
+    with pytest.raises(A.AnpdError) as e:
+        A.anpd_kv_truncate(c1.kv, 0, 10)                               # cannot grow
+    assert e.value.status == A.ERR_RANGE
+    with pytest.raises(A.AnpdError) as e:
+        A.anpd_prefill(c1.m, c1.kv, list(range(600)))                  # longer than the cache
+    assert e.value.status in (A.ERR_STATE, A.ERR_CAPACITY)

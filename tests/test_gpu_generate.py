@@ -1,0 +1,178 @@
+"""Algorithm 1 on the GPU: the ANPD token stream is bit-identical to the same library's greedy
+stream (losslessness), agrees with the oracle's greedy stream wherever the oracle's deciding
+margin is large enough, and its per-step drafts / accepted lengths follow the oracle's."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import agree_until_low_margin, as_bf16_values, gpu_model, oracle_greedy_with_margins, require_gpu
+from oracle.anpd import anpd_generate as oracle_anpd
+from oracle.decoder import Decoder
+from oracle.mln import MLN
+from workloads import WORKLOADS, ModelShape, make_prompts, make_weights, markov_prompt, periodic_prompt
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def A():
+    require_gpu()
+    from paper_2404_08698_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def c1(A):
+    wl = WORKLOADS["C1"]
+    w = make_weights(wl.shape, wl.weight_seed, wl.weights_bf16)
+    m = gpu_model(A, wl.shape, w)
+    kv = A.anpd_kv_create(m, 512)
+    yield wl, w, m, kv
+    A.anpd_kv_destroy(kv)
+    A.anpd_model_destroy(m)
+
+
+def test_c1_anpd_equals_greedy_equals_oracle(A, c1):
+    wl, w, m, kv = c1
+    prompt = make_prompts(wl)[0]
+    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, 512)
+    try:
+        out, st = A.anpd_generate(m, kv, ctx, prompt, wl.max_new, wl.K)
+        ref, st0 = A.anpd_generate(m, kv, ctx, prompt, wl.max_new, 0)
+        assert np.array_equal(out, ref)                                 # losslessness, bit for bit
+        assert st0["steps"] == wl.max_new and st0["drafted"] == 0
+        # progress: each step commits 1..K+1 tokens; generated = steps + accepted
+        assert st["generated"] == st["steps"] + st["accepted"] and st["generated"] >= wl.max_new
+        assert sum(st["hist_accepted"]) == st["steps"] and sum(st["hist_accepted"][wl.K + 1:]) == 0
+        assert st["accepted"] == sum(i * h for i, h in enumerate(st["hist_accepted"]))
+        dec = Decoder(wl.shape, as_bf16_values(w), torch.float64)
+        want, margins = oracle_greedy_with_margins(dec, prompt.tolist(), wl.max_new)
+        n = agree_until_low_margin(ref, want, margins)
+        assert n >= 8, n
+        if n == wl.max_new:
+            # same stream: the oracle's Algorithm 1 must have taken the same steps
+            _, ost, _ = oracle_anpd(dec, prompt.tolist(), wl.max_new, wl.K, n_max=wl.n_max)
+            assert st["steps"] == ost.steps and st["accepted"] == ost.accepted and st["drafted"] == ost.drafted
+            assert st["hist_accepted"] == ost.hist_accepted
+    finally:
+        A.anpd_ngram_destroy(ctx)
+
+
+def test_tables_after_generate_match_oracle_on_the_generated_stream(A, c1):
+    wl, w, m, kv = c1
+    prompt = make_prompts(wl)[0]
+    ctx = A.anpd_ngram_create(2, 4, 512)
+    try:
+        ref, _ = A.anpd_generate(m, kv, ctx, prompt, 48, 0)             # greedy, a little longer
+        out, st = A.anpd_generate(m, kv, ctx, prompt, 40, 5)
+        assert np.array_equal(out, ref[:40])
+        n_ctx = A.anpd_ngram_len(ctx)
+        assert n_ctx == len(prompt) + st["generated"] and 40 <= st["generated"] <= 45
+        assert A.anpd_kv_len(kv) == n_ctx - 1                           # the last token is not in the cache yet
+        # the loop may overshoot max_new; by losslessness the context holds the greedy stream
+        committed = prompt.tolist() + ref[:st["generated"]].tolist()
+        assert A.anpd_ngram_draft(ctx, 0) == []                         # folds the last step's tokens
+        mln = MLN(2, 4)
+        mln.initialize(committed)
+        for n in (2, 3, 4):
+            assert A.anpd_ngram_dump(ctx, n) == mln.dump(n)
+        assert A.anpd_ngram_draft(ctx, 5) == mln.draft(5)
+    finally:
+        A.anpd_ngram_destroy(ctx)
+
+
+@pytest.mark.parametrize("K,N,policy", [(1, 2, 0), (3, 2, 1), (5, 5, 0), (7, 8, 0), (7, 3, 1), (2, 6, 0)])
+def test_losslessness_over_K_N_policy(A, K, N, policy):
+    shape = ModelShape(2, 128, 4, 2, 64, 200, 300)
+    w = make_weights(shape, 21, False, std=0.08)
+    m = gpu_model(A, shape, w)
+    kv = A.anpd_kv_create(m, 256)
+    ctx = A.anpd_ngram_create(2, N, 256, policy)
+    try:
+        base = periodic_prompt(30, 6, shape.vocab, 4)
+        prompt = np.concatenate([base, markov_prompt(30, shape.vocab, 2, 8), base[:13]])
+        ref, _ = A.anpd_generate(m, kv, ctx, prompt, 48, 0)
+        out, st = A.anpd_generate(m, kv, ctx, prompt, 48, K)
+        assert np.array_equal(out, ref)
+        assert st["generated"] == st["steps"] + st["accepted"]
+        assert st["drafted"] <= K * st["steps"]
+    finally:
+        A.anpd_ngram_destroy(ctx)
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(m)
+
+
+def test_cyclic_copy_model_accepts_every_draft(A):
+    """A decoder whose attention and FFN outputs are zero and whose LM head reads the embedding of
+    the successor in a fixed cycle: greedy output is that cycle (closed form), and once a period has
+    been seen every draft is accepted."""
+    V, d = 16, 64
+    shape = ModelShape(1, d, 1, 1, 64, 64, V)
+    w = make_weights(shape, 3, False, std=0.05)
+    w["l0.wo"].zero_()
+    w["l0.w_down"].zero_()
+    e = torch.zeros(V, d)
+    for t in range(V):
+        e[t, t] = 1.0
+    w["embed"] = e
+    perm = [(t + 1) % 5 if t < 5 else 0 for t in range(V)]               # cycle 0 1 2 3 4
+    lm = torch.zeros(V, d)
+    for t in range(V):
+        lm[perm[t], t] = 1.0                                             # logits[perm[t]] = h[t]
+    w["lm_head"] = lm
+    m = gpu_model(A, shape, w)
+    kv = A.anpd_kv_create(m, 256)
+    ctx = A.anpd_ngram_create(2, 3, 256)
+    try:
+        prompt = [t % 5 for t in range(12)]
+        K, M = 4, 40
+        out, st = A.anpd_generate(m, kv, ctx, prompt, M, K)
+        assert out.tolist() == [(12 + i) % 5 for i in range(M)]
+        assert st["hist_accepted"][K] == st["steps"] and st["steps"] == -(-M // (K + 1))
+    finally:
+        A.anpd_ngram_destroy(ctx)
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(m)
+
+
+def test_batch_equals_independent_runs(A):
+    shape = ModelShape(2, 128, 4, 4, 64, 200, 300)
+    w = make_weights(shape, 9, False, std=0.08)
+    m = gpu_model(A, shape, w)
+    B, plen, M, K = 3, 70, 30, 4
+    prompts = np.stack([np.concatenate([markov_prompt(35, shape.vocab, 2, 50 + b)] * 2) for b in range(B)])
+    kv1 = A.anpd_kv_create(m, 256, 1)
+    kvb = A.anpd_kv_create(m, 256, B, True)
+    ctxs = [A.anpd_ngram_create(2, 4, 256) for _ in range(B)]
+    try:
+        singles = [A.anpd_generate(m, kv1, ctxs[0], prompts[b], M, K) for b in range(B)]
+        outs, stats = A.anpd_generate_batch(m, kvb, ctxs, prompts, M, K)
+        for b in range(B):
+            assert np.array_equal(outs[b], singles[b][0]), b
+            for k in ("steps", "drafted", "accepted", "generated", "hist_accepted"):
+                assert stats[b][k] == singles[b][1][k], (b, k)
+        greedy, _ = A.anpd_generate_batch(m, kvb, ctxs, prompts, M, 0)
+        assert np.array_equal(greedy, outs)
+    finally:
+        for c in ctxs:
+            A.anpd_ngram_destroy(c)
+        A.anpd_kv_destroy(kv1)
+        A.anpd_kv_destroy(kvb)
+        A.anpd_model_destroy(m)
+
+
+def test_generate_error_paths(A, c1):
+    wl, w, m, kv = c1
+    ctx = A.anpd_ngram_create(2, 3, 128)
+    try:
+        with pytest.raises(A.AnpdError) as e:
+            A.anpd_generate(m, kv, ctx, list(range(100)), 64, 4)         # context too small
+        assert e.value.status == A.ERR_CAPACITY
+        with pytest.raises(A.AnpdError) as e:
+            A.anpd_generate(m, kv, ctx, [1, 2, 3], 8, 8)                 # K > 7
+        assert e.value.status == A.ERR_RANGE
+        with pytest.raises(A.AnpdError) as e:
+            A.anpd_generate(m, kv, ctx, [1, 2, 5000], 8, 2)              # token out of vocab
+        assert e.value.status == A.ERR_RANGE
+    finally:
+        A.anpd_ngram_destroy(ctx)
