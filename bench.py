@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the ANPD draft-and-verify path on B200.
+
+One "step" is one whole run of the hot path on the workload: Initialize + prefill + the
+draft-and-verify loop until max_new tokens are out (anpd_generate).  The headline value is
+generated tokens per second of that run; the same build's plain greedy decode (K = 0, same
+kernels) is timed beside it, and a verify-step microbenchmark gives the achieved fraction of the
+HBM roofline.  Prints ONE JSON line on rank 0.
+
+  python bench.py                       # 1 GPU, 7B shape (workload C3)
+  python bench.py --workload C2         # 1.1B shape
+  python bench.py --impl reference      # the CPU oracle on the host cores, bounded sample
+  torchrun ... bench.py --gpus N        # N independent replicas (the path does not shard)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from workloads import WORKLOADS, make_prompts, make_weights, tensor_shapes
+
+METRIC = "tokens_per_s_bs1_anpd"
+UNIT = "tokens/s"
+HBM_NOMINAL_GBS = 8000.0          # the roofline the target is stated against
+HBM_FALLBACK_GBS = 6650.0         # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
+
+
+def measured_hbm_peak() -> tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons = [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    out["sm_max_mhz"] = float(f[1])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+        out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_sample(wl, weights_cpu, prompt, sample_prompt: int, sample_new: int) -> dict:
+    """Times the CPU oracle (as it stands) on a bounded sample of the workload."""
+    from oracle.anpd import anpd_generate as oracle_anpd
+    from oracle.decoder import Decoder
+    dec = Decoder(wl.shape, weights_cpu, torch.float64)
+    t0 = time.perf_counter()
+    out, st, _ = oracle_anpd(dec, prompt[:sample_prompt].tolist(), sample_new, wl.K, n_max=wl.n_max, n_min=wl.n_min)
+    dt = time.perf_counter() - t0
+    return {"value": len(out) / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"oracle Algorithm 1 (fp64 torch CPU ops) on the first {sample_prompt} prompt tokens of {wl.name}, "
+                      f"{sample_new} new tokens, N={wl.n_max}, K={wl.K}: {st.steps} verify forwards + 1 prefill in {dt:.1f} s"}
+
+
+def run_reference(args) -> None:
+    """--impl reference: the oracle on the host cores, same config / metric / unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = WORKLOADS[args.workload]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = make_weights(wl.shape, wl.weight_seed, wl.weights_bf16, device=dev)
+    w = {k: v.cpu() for k, v in w.items()}
+    prompt = make_prompts(wl)[0]
+    big = wl.shape.streamed_params > 3e9
+    sp, sn = (16, 2) if big else ((64, 8) if wl.shape.streamed_params > 1e8 else (wl.prompt_len, wl.max_new))
+    for _ in range(args.warmup):
+        oracle_sample(wl, w, prompt, sp, 1)
+    t0 = time.perf_counter()
+    res = [oracle_sample(wl, w, prompt, sp, sn) for _ in range(args.steps)]
+    dt = time.perf_counter() - t0
+    value = args.steps * sn / dt
+    cpu = dict(res[-1])
+    cpu["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name} (bounded sample: first {sp} prompt tokens, {sn} new tokens per step)",
+                   "n_max": wl.n_max, "K": wl.K},
+        "cpu_baseline": cpu,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--verify-iters", type=int, default=40)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2404_08698_b200 import binding as A, build
+    build.build()
+
+    wl = WORKLOADS[args.workload]
+    shape = wl.shape
+    stream = torch.cuda.Stream()
+    t_setup = time.perf_counter()
+    w = make_weights(shape, wl.weight_seed, wl.weights_bf16, device="cuda")
+    torch.cuda.synchronize()
+    model = A.anpd_model_create(shape, [w[n] for n, _ in tensor_shapes(shape)], stream.cuda_stream)
+    want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
+    w_cpu = {k: v.cpu() for k, v in w.items()} if want_cpu else None
+    del w
+    torch.cuda.empty_cache()
+    max_len = wl.prompt_len + wl.max_new + 64
+    kv = A.anpd_kv_create(model, max_len)
+    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, stream.cuda_stream)
+    prompt = make_prompts(wl)[0]
+    prompt_dev = torch.from_numpy(prompt).cuda()
+    out_dev = torch.zeros(wl.max_new, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    t_setup = time.perf_counter() - t_setup
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+
+    def timed(K: int, steps: int, warmup: int):
+        """Device time (CUDA events on the library's stream) of `steps` generate runs."""
+        st = None
+        for _ in range(warmup):
+            st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+        e1.record(stream)
+        barrier()
+        return e0.elapsed_time(e1) / 1e3, st
+
+    # ---- headline: ANPD generate, inputs resident on the device --------------------------------
+    A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, wl.K, out_dev)        # first-touch
+    sampler = ClockSampler(local)
+    A.anpd_launch_count(True)
+    for _ in range(args.warmup):
+        A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, wl.K, out_dev)
+    launches_warm = A.anpd_launch_count(True)
+    sampler.start()
+    t_anpd, st_anpd = timed(wl.K, args.steps, 0)
+    clocks = sampler.stop()
+    launches = A.anpd_launch_count(True)
+    anpd_tokens = out_dev.cpu().numpy().copy()
+    if dist is not None:
+        t = torch.tensor([t_anpd], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_anpd = float(t.item())
+    value = world * args.steps * wl.max_new / t_anpd
+
+    # ---- the same build's plain greedy decode --------------------------------------------------
+    t_greedy, st_greedy = timed(0, args.steps, 1)
+    greedy_tokens = out_dev.cpu().numpy().copy()
+    lossless = bool(np.array_equal(anpd_tokens, greedy_tokens))
+    greedy_tps = args.steps * wl.max_new / t_greedy
+
+    # ---- end to end through the host-buffer call -------------------------------------------------
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        out_host, _ = A.anpd_generate(model, kv, ctx, prompt, wl.max_new, wl.K)
+    torch.cuda.synchronize()
+    t_e2e = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([t_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e = float(t.item())
+    e2e = {"value": world * args.steps * wl.max_new / t_e2e, "unit": UNIT,
+           "h2d_bytes_per_step": int(prompt.nbytes), "d2h_bytes_per_step": int(out_host.nbytes)}
+
+    # ---- verify-step microbenchmark at the end-of-prompt KV length ------------------------------
+    A.anpd_kv_truncate(kv, 0, 0)
+    first = A.anpd_prefill(model, kv, prompt)
+    P = A.anpd_kv_len(kv)
+    draft = [int(x) for x in prompt[:wl.K]]
+    A.anpd_verify_stage(model, kv, [first], [draft])
+    for _ in range(3):
+        A.anpd_verify_enqueue(model, kv)
+        A.anpd_kv_truncate(kv, 0, P)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.verify_iters):
+        A.anpd_verify_enqueue(model, kv)
+        A.anpd_kv_truncate(kv, 0, P)
+    e1.record(stream)
+    barrier()
+    ms_verify = e0.elapsed_time(e1) / args.verify_iters
+    step_bytes = shape.streamed_params * 2 + shape.kv_bytes_per_token * (P + A.ROWS)
+    verify_gbs = step_bytes / (ms_verify * 1e-3) / 1e9
+
+    # ---- dominant kernel (the weight-streaming GEMM), per-launch device time ----------------------
+    A.anpd_profile_enable(model, True)
+    A.anpd_profile_read(model, True)
+    for _ in range(5):
+        A.anpd_verify_enqueue(model, kv)
+        A.anpd_kv_truncate(kv, 0, P)
+    prof = A.anpd_profile_read(model, True)
+    A.anpd_profile_enable(model, False)
+    peak, peak_kind = measured_hbm_peak()
+    gemm_gbs = prof["gemm_bytes"] / (prof["ms_gemm"] * 1e-3) / 1e9 if prof["ms_gemm"] > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections + LM head)",
+                "achieved": gemm_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": gemm_gbs / peak, "traffic": None,
+                "launches": prof["n_gemm"], "avg_launch_us": prof["ms_gemm"] * 1e3 / max(prof["n_gemm"], 1),
+                "bytes_per_launch": prof["gemm_bytes"] / max(prof["n_gemm"], 1),
+                "step_share": {"gemm_ms": prof["ms_gemm"] / 5, "attn_ms": prof["ms_attn"] / 5,
+                               "other_ms": prof["ms_other"] / 5}}
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t_anpd / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: {shape.n_layers}L d{shape.d_model} {shape.n_q_heads}q/{shape.n_kv_heads}kv x{shape.head_dim} "
+                               f"ffn{shape.d_ffn} vocab{shape.vocab}, prompt {wl.prompt_len}, {wl.max_new} new tokens, batch 1",
+                   "n_max": wl.n_max, "K": wl.K, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "l2": "inputs (weights) far larger than L2; no flush", "step": "one anpd_generate run (prefill + decode loop)"},
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+        "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline,
+        "anpd": {"tokens_per_s": args.steps * wl.max_new / t_anpd if world == 1 else value / world,
+                 "decode_tokens_per_s": st_anpd["generated"] / (st_anpd["ms_decode"] * 1e-3),
+                 "ms_prefill": st_anpd["ms_prefill"], "ms_decode": st_anpd["ms_decode"], "steps": st_anpd["steps"],
+                 "mean_accepted_per_step": st_anpd["accepted"] / max(st_anpd["steps"], 1),
+                 "hit_ratio_alpha": st_anpd["accepted"] / max(st_anpd["drafted"], 1),
+                 "hist_accepted": st_anpd["hist_accepted"]},
+        "greedy": {"tokens_per_s": greedy_tps, "decode_tokens_per_s": st_greedy["generated"] / (st_greedy["ms_decode"] * 1e-3),
+                   "ms_prefill": st_greedy["ms_prefill"], "ms_decode": st_greedy["ms_decode"]},
+        "speedup_vs_greedy": (args.steps * wl.max_new / t_anpd) / greedy_tps if world == 1 else None,
+        "decode_speedup_vs_greedy": st_greedy["ms_decode"] / st_anpd["ms_decode"] * st_anpd["generated"] / st_greedy["generated"],
+        "anpd_equals_greedy": lossless,
+        "verify_step": {"kv_len": P, "rows": A.ROWS, "ms": ms_verify, "bytes": step_bytes, "gbs": verify_gbs,
+                        "frac_of_8TBs": verify_gbs / HBM_NOMINAL_GBS, f"frac_of_{peak_kind}_copy": verify_gbs / peak},
+        "setup_s": t_setup,
+    }
+    if want_cpu:
+        big = shape.streamed_params > 3e9
+        sp, sn = (16, 2) if big else ((64, 8) if shape.streamed_params > 1e8 else (wl.prompt_len, wl.max_new))
+        result["cpu_baseline"] = oracle_sample(wl, w_cpu, prompt, sp, sn)
+    if rank == 0:
+        print(json.dumps(result))
+    A.anpd_ngram_destroy(ctx)
+    A.anpd_kv_destroy(kv)
+    A.anpd_model_destroy(model)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

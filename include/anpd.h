@@ -204,6 +204,13 @@ anpd_status anpd_generate(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const int
                           int prompt_len, int max_new, int K, int32_t* out, int* n_out,
                           anpd_stats* stats);
 
+/* anpd_generate with the prompt and the output in DEVICE memory (int32 on the model's device):
+ * no host buffer is touched except the few bytes of loop control read back per step.  Token ids
+ * are validated on the device (ANPD_ERR_RANGE after the fact). */
+anpd_status anpd_generate_dev(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const int32_t* prompt_dev,
+                              int prompt_len, int max_new, int K, int32_t* out_dev, int* n_out,
+                              anpd_stats* stats);
+
 /* Batch of independent sequences sharing one weight stream per step: ctxs[B], prompts
  * [B * prompt_len] (equal lengths), out [B * max_new], stats [B] or NULL. */
 anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* ctxs,
@@ -215,6 +222,13 @@ anpd_status anpd_profile_enable(anpd_model* m, int on); /* on: time every launch
 anpd_status anpd_profile_read(anpd_model* m, anpd_profile* out, int reset);
 /* Number of kernel launches issued by this library since the last reset (all handles). */
 long long anpd_launch_count(int reset);
+
+/* Test hook for the projections inside LLM(drafts) (Section 3.1, "Verification"):
+ * out[rows][N] = A[rows][K] x W[N][K]^T through the library's weight-streaming GEMM kernel, on
+ * the current device and the default stream.  W: N*K bf16 bit patterns (host); A: rows*K fp32
+ * (host), rows a multiple of 8 and at most 128; K a multiple of 8.  plain != 0 selects the
+ * reference kernel the tensor-core kernel is cross-checked against. */
+anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a, int rows, float* out, int plain);
 
 const char* anpd_status_string(anpd_status s);
 

@@ -86,10 +86,13 @@ SIGNATURES = {
     "anpd_verify_enqueue": (C.c_int, [_P, _P]),
     "anpd_verify_result": (C.c_int, [_P, _P, _IP, _I32P]),
     "anpd_generate": (C.c_int, [_P, _P, _P, _I32P, C.c_int, C.c_int, C.c_int, _I32P, _IP, C.POINTER(Stats)]),
+    "anpd_generate_dev": (C.c_int, [_P, _P, _P, _P, C.c_int, C.c_int, C.c_int, _P, _IP, C.POINTER(Stats)]),
     "anpd_generate_batch": (C.c_int, [_P, _P, C.POINTER(_P), _I32P, C.c_int, C.c_int, C.c_int, _I32P, C.POINTER(Stats)]),
     "anpd_profile_enable": (C.c_int, [_P, C.c_int]),
     "anpd_profile_read": (C.c_int, [_P, C.POINTER(Profile), C.c_int]),
     "anpd_launch_count": (C.c_longlong, [C.c_int]),
+    "anpd_debug_gemm": (C.c_int, [C.POINTER(C.c_uint16), C.c_int, C.c_int, C.POINTER(C.c_float), C.c_int,
+                                  C.POINTER(C.c_float), C.c_int]),
     "anpd_status_string": (C.c_char_p, [C.c_int]),
 }
 
@@ -295,6 +298,15 @@ def anpd_generate(m: int, kv: int, ctx: int, prompt, max_new: int, K: int) -> tu
     return out[:n_out.value], st.as_dict()
 
 
+def anpd_generate_dev(m: int, kv: int, ctx: int, prompt_dev, max_new: int, K: int, out_dev) -> dict:
+    """prompt_dev / out_dev: int32 CUDA tensors (out_dev holds at least max_new elements)."""
+    n_out = C.c_int()
+    st = Stats()
+    _check(lib().anpd_generate_dev(_P(m), _P(kv), _P(ctx), _P(prompt_dev.data_ptr()), prompt_dev.numel(), max_new, K,
+                                   _P(out_dev.data_ptr()), C.byref(n_out), C.byref(st)), "anpd_generate_dev")
+    return st.as_dict()
+
+
 def anpd_generate_batch(m: int, kv: int, ctxs: list[int], prompts, max_new: int, K: int):
     p = np.ascontiguousarray(np.asarray(prompts, dtype=np.int32))
     B, plen = p.shape
@@ -318,3 +330,16 @@ def anpd_profile_read(m: int, reset: bool = True) -> dict:
 
 def anpd_launch_count(reset: bool = False) -> int:
     return int(lib().anpd_launch_count(int(reset)))
+
+
+def anpd_debug_gemm(w_bf16, a, plain: bool = False) -> np.ndarray:
+    """w_bf16: torch bf16 CPU tensor [N, K]; a: fp32 array [rows, K].  Returns out [rows, N] fp32."""
+    import torch
+    N, K = w_bf16.shape
+    wb = np.ascontiguousarray(w_bf16.contiguous().view(torch.int16).numpy().view(np.uint16))
+    a = np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+    rows = a.shape[0]
+    out = np.zeros((rows, N), dtype=np.float32)
+    _check(lib().anpd_debug_gemm(wb.ctypes.data_as(C.POINTER(C.c_uint16)), N, K, a.ctypes.data_as(C.POINTER(C.c_float)), rows,
+                                 out.ctypes.data_as(C.POINTER(C.c_float)), int(plain)), "anpd_debug_gemm")
+    return out

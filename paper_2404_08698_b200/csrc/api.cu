@@ -106,6 +106,50 @@ bool have_device() {
 
 }  // namespace
 
+// GEMM plans (how each matrix shape is cut across the SMs) and the TMA views of the weights.
+static anpd_status model_make_plans(anpd_model* m) {
+    const anpd_model_config& c = m->cfg;
+    int dev = 0, sms = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    m->num_sms = sms;
+    m->plain_gemm = std::getenv("ANPD_PLAIN_GEMM") != nullptr;
+    const int shapes[GK_COUNT][2] = {{m->nqkv, c.d_model}, {c.d_model, m->dq}, {2 * c.d_ffn, c.d_model}, {c.d_model, c.d_ffn},
+                                     {c.vocab, c.d_model}};
+    size_t ints = 0;
+    int max_tiles = 0;
+    m->max_segs = 1;
+    for (int k = 0; k < GK_COUNT; ++k) {
+        gemm_make_plan(&m->plan[k], shapes[k][0], shapes[k][1], sms);
+        ints += 2 * (size_t)m->plan[k].m_tiles;
+        max_tiles = std::max(max_tiles, m->plan[k].m_tiles);
+        m->max_segs = std::max(m->max_segs, m->plan[k].max_segs);
+    }
+    ints += max_tiles;
+    std::vector<int> host(ints);
+    CUDA_TRY(cudaMalloc((void**)&m->d_plan_tables, ints * sizeof(int)));
+    size_t off = 0;
+    for (int k = 0; k < GK_COUNT; ++k) {
+        GemmPlan& p = m->plan[k];
+        p.d_first_cta = m->d_plan_tables + off;
+        std::copy(p.first_cta.begin(), p.first_cta.end(), host.begin() + off); off += p.m_tiles;
+        p.d_seg_count = m->d_plan_tables + off;
+        std::copy(p.seg_count.begin(), p.seg_count.end(), host.begin() + off); off += p.m_tiles;
+    }
+    m->d_ones = m->d_plan_tables + off;
+    for (int i = 0; i < max_tiles; ++i) host[off + i] = 1;
+    CUDA_TRY(cudaMemcpy(m->d_plan_tables, host.data(), ints * sizeof(int), cudaMemcpyHostToDevice));
+    for (int l = 0; l < c.n_layers; ++l) {
+        LayerW& w = m->layers[l];
+        ANPD_TRY(make_tmap_bf16(&w.map[GK_QKV], w.wqkv, m->nqkv, c.d_model, 128, true));
+        ANPD_TRY(make_tmap_bf16(&w.map[GK_O], w.wo, c.d_model, m->dq, 128, true));
+        ANPD_TRY(make_tmap_bf16(&w.map[GK_GU], w.wgu, 2 * c.d_ffn, c.d_model, 128, true));
+        ANPD_TRY(make_tmap_bf16(&w.map[GK_DOWN], w.wd, c.d_model, c.d_ffn, 128, true));
+    }
+    ANPD_TRY(make_tmap_bf16(&m->map_lm, m->lm_head, c.vocab, c.d_model, 128, true));
+    return ANPD_OK;
+}
+
 extern "C" {
 
 const char* anpd_status_string(anpd_status s) {
@@ -193,7 +237,9 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     m->final_norm = (const float*)put(weights[t++], d, false, b_norm);
     m->lm_head = (const bf16*)put(weights[t++], V * d, true, b_embed);
     if (rc == ANPD_OK && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
-    if (rc != ANPD_OK) { cudaFree(m->slab); delete m; return rc; }
+    m->d_plan_tables = nullptr;
+    if (rc == ANPD_OK) rc = model_make_plans(m);
+    if (rc != ANPD_OK) { cudaFree(m->d_plan_tables); cudaFree(m->slab); delete m; return rc; }
     *out = m;
     return ANPD_OK;
 }
@@ -201,6 +247,7 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
 anpd_status anpd_model_destroy(anpd_model* m) {
     if (!m) return ANPD_ERR_ARG;
     cudaStreamSynchronize(m->stream);
+    cudaFree(m->d_plan_tables);
     cudaFree(m->slab);
     delete m;
     return ANPD_OK;
@@ -210,7 +257,7 @@ anpd_status anpd_model_destroy(anpd_model* m) {
 // KV cache + workspace
 // ---------------------------------------------------------------------------------------------
 anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shuffle_pages, anpd_kv** out) {
-    if (!cm || !out || max_len < ANPD_ROWS || batch < 1 || batch > 64) return ANPD_ERR_ARG;
+    if (!cm || !out || max_len < ANPD_ROWS || batch < 1 || batch > 16) return ANPD_ERR_ARG;
     anpd_model* m = const_cast<anpd_model*>(cm);
     const anpd_model_config& c = m->cfg;
     anpd_kv* kv = new (std::nothrow) anpd_kv();
@@ -224,7 +271,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     Workspace& ws = kv->ws;
     ws.r_max = std::max(PREFILL_ROWS, batch * ANPD_ROWS);
     ws.n_max_out = std::max(std::max(m->nqkv, 2 * c.d_ffn), std::max(c.d_model, c.vocab));
-    ws.splits_max = 1;
+    ws.splits_max = m->max_segs;
     ws.amax_blocks = (c.vocab + 1023) / 1024;
     const size_t R = ws.r_max, d = c.d_model, F = c.d_ffn, V = c.vocab, hd = c.head_dim, half = hd / 2;
     const size_t pool = (size_t)c.n_layers * kv->total_pages * c.n_kv_heads * KV_PAGE * hd * 2;
@@ -245,6 +292,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&ws.attn_m, n_part * 4}, {(void**)&ws.attn_l, n_part * 4}, {(void**)&ws.attn_o, n_part * hd * 4},
         {(void**)&ws.logits, R * V * 4},
         {(void**)&ws.amax_val, R * ws.amax_blocks * 4}, {(void**)&ws.amax_idx, R * ws.amax_blocks * 4},
+        {(void**)&ws.gemm_err, 256},
     };
     size_t total = 0;
     for (const Item& it : items) total += up256(it.bytes);
@@ -255,6 +303,24 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     const size_t pinned_bytes = sizeof(SeqState) * (size_t)batch + 64 * sizeof(int) * (size_t)batch + 256;
     if (cudaMallocHost((void**)&kv->h_seq, pinned_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(kv->slab); delete kv; return ANPD_ERR_OOM; }
     kv->h_small = (int*)((char*)kv->h_seq + sizeof(SeqState) * (size_t)batch);
+
+    // TMA views of the GEMM inputs: decode rows (batch * 8) and prefill rows, each padded to the MMA's N
+    {
+        const int mode_rows[2] = {batch * ANPD_ROWS, PREFILL_ROWS};
+        anpd_status rc = ANPD_OK;
+        for (int md = 0; md < 2 && rc == ANPD_OK; ++md) {
+            const int rows = mode_rows[md], nb = (rows + 15) / 16 * 16;
+            ws.nb[md] = nb;
+            struct { CUtensorMap* maps; const bf16* hi; const bf16* lo; int K; } bufs[3] = {
+                {ws.map_h[md], ws.h_hi, ws.h_lo, c.d_model}, {ws.map_ao[md], ws.ao_hi, ws.ao_lo, m->dq}, {ws.map_act[md], ws.act_hi, ws.act_lo, c.d_ffn}};
+            for (auto& bdesc : bufs) {
+                // rows beyond the tensor's extent are zero-filled by the copy engine
+                if (rc == ANPD_OK) rc = make_tmap_bf16(&bdesc.maps[0], bdesc.hi, rows, bdesc.K, nb, false);
+                if (rc == ANPD_OK) rc = make_tmap_bf16(&bdesc.maps[1], bdesc.lo, rows, bdesc.K, nb, false);
+            }
+        }
+        if (rc != ANPD_OK) { cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv; return rc; }
+    }
 
     // page table: identity, or a fixed permutation of the physical pages
     std::vector<int> pt(kv->total_pages);
@@ -335,7 +401,7 @@ static anpd_status kv_reset(anpd_kv* kv, const int* stop_at) {
 // ---------------------------------------------------------------------------------------------
 static anpd_status prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, const int32_t* prompt, int prompt_len,
                                    const NgramDev* d_ctxs) {
-    CUDA_TRY(cudaMemcpyAsync(kv->d_prompt, prompt, sizeof(int) * (size_t)prompt_len, cudaMemcpyHostToDevice, m->stream));
+    CUDA_TRY(cudaMemcpyAsync(kv->d_prompt, prompt, sizeof(int) * (size_t)prompt_len, cudaMemcpyDefault, m->stream));
     for (int start = 0; start < prompt_len; start += PREFILL_ROWS) {
         const int n = std::min(PREFILL_ROWS, prompt_len - start);
         const int rows = (n + ANPD_ROWS - 1) / ANPD_ROWS * ANPD_ROWS;
@@ -348,9 +414,15 @@ static anpd_status prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, const in
 }
 
 static anpd_status read_seqs(anpd_kv* kv) {
+    int* h_err = kv->h_small + 48 * kv->batch;
     CUDA_TRY(cudaMemcpyAsync(kv->h_seq, kv->seq, sizeof(SeqState) * (size_t)kv->batch, cudaMemcpyDeviceToHost, kv->m->stream));
+    CUDA_TRY(cudaMemcpyAsync(h_err, kv->ws.gemm_err, sizeof(int), cudaMemcpyDeviceToHost, kv->m->stream));
     CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
     for (int b = 0; b < kv->batch; ++b) kv->h_kv_len[b] = kv->h_seq[b].kv_len;
+    if (*h_err != 0) {
+        std::snprintf(g_last_error, sizeof(g_last_error), "a GEMM kernel gave up waiting (code %d)", *h_err);
+        return ANPD_ERR_CUDA;
+    }
     return ANPD_OK;
 }
 
@@ -463,20 +535,23 @@ anpd_status anpd_verify_logits(anpd_model* m, anpd_kv* kv, int32_t last_tok, con
 // ---------------------------------------------------------------------------------------------
 // Algorithm 1
 // ---------------------------------------------------------------------------------------------
-anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* ctxs, const int32_t* prompts,
-                                int prompt_len, int max_new, int K, int32_t* out, anpd_stats* stats) {
+static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* ctxs, const int32_t* prompts,
+                                 int prompt_len, int max_new, int K, int32_t* out, anpd_stats* stats, bool on_device) {
     if (!m || !kv || kv->m != m || !ctxs || !prompts || !out || prompt_len < 1 || max_new < 1) return ANPD_ERR_ARG;
     if (K < 0 || K > ANPD_K_MAX) return ANPD_ERR_RANGE;
     const int B = kv->batch;
     cudaStream_t st = m->stream;
     for (int b = 0; b < B; ++b) {
         if (!ctxs[b] || ctxs[b]->stream != st) return ANPD_ERR_ARG;
-        if (prompt_len + max_new + ANPD_ROWS > ctxs[b]->h.max_ctx) return ANPD_ERR_CAPACITY;
+        if (prompt_len + max_new + 1 + ANPD_ROWS > ctxs[b]->h.max_ctx) return ANPD_ERR_CAPACITY;
     }
     if (prompt_len + max_new + 2 * ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
-    for (size_t i = 0; i < (size_t)B * prompt_len; ++i) if (prompts[i] < 0 || prompts[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+    if (!on_device)
+        for (size_t i = 0; i < (size_t)B * prompt_len; ++i) if (prompts[i] < 0 || prompts[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
 
-    std::vector<int> stop(B, prompt_len + max_new);
+    // Algorithm 1 tests length(O) < M at the top of the loop, where O receives the token confirmed by
+    // the previous step; the context holds that pending token too, hence the + 1
+    std::vector<int> stop(B, prompt_len + max_new + 1);
     ANPD_TRY(kv_reset(kv, stop.data()));
     std::vector<NgramDev> hd(B);
     for (int b = 0; b < B; ++b) {
@@ -495,7 +570,7 @@ anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* c
         for (int b = 0; b < B; ++b) {
             anpd_ngram* c = ctxs[b];
             CUDA_TRY(cudaMemcpyAsync(c->h.tokens, prompts + (size_t)b * prompt_len, sizeof(int) * (size_t)prompt_len,
-                                     cudaMemcpyHostToDevice, st));
+                                     cudaMemcpyDefault, st));
             kv->h_small[2 * b] = prompt_len; kv->h_small[2 * b + 1] = (K > 0) ? prompt_len : 0;
             CUDA_TRY(cudaMemcpyAsync(c->h.state, kv->h_small + 2 * b, 2 * sizeof(int), cudaMemcpyHostToDevice, st));
             if (K > 0) ANPD_TRY(ngram_enqueue_bulk(c, 0, prompt_len, &m->prof));
@@ -528,7 +603,7 @@ anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* c
         cudaEventElapsedTime(&ms_d, e1, e2);
         for (int b = 0; b < B && rc == ANPD_OK; ++b) {
             if (cudaMemcpy(out + (size_t)b * max_new, ctxs[b]->h.tokens + prompt_len, sizeof(int) * (size_t)max_new,
-                           cudaMemcpyDeviceToHost) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; break; }
+                           cudaMemcpyDefault) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; break; }
             int nst[2] = {0, 0};
             if (cudaMemcpy(nst, ctxs[b]->h.state, 2 * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = ANPD_ERR_CUDA; break; }
             const int nt = nst[0];
@@ -537,10 +612,10 @@ anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* c
             if (stats) {
                 const SeqState& s = kv->h_seq[b];
                 anpd_stats& o = stats[b];
-                o.steps = s.steps; o.drafted = s.drafted; o.accepted = s.accepted; o.generated = nt - prompt_len;
+                o.steps = s.steps; o.drafted = s.drafted; o.accepted = s.accepted; o.generated = nt - prompt_len - 1;
                 for (int i = 0; i < 8; ++i) o.hist_accepted[i] = s.hist[i];
                 o.ms_prefill = ms_p; o.ms_decode = ms_d;
-                const double mean_kv = prompt_len + 0.5 * (nt - prompt_len);
+                const double mean_kv = prompt_len + 0.5 * (nt - prompt_len - 1);
                 const anpd_model_config& c = m->cfg;
                 o.bytes_per_step = m->streamed_bytes + B * mean_kv * (2.0 * c.n_layers * c.n_kv_heads * c.head_dim * 2.0);
             }
@@ -550,13 +625,92 @@ anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* c
     return rc;
 }
 
+anpd_status anpd_generate_batch(anpd_model* m, anpd_kv* kv, anpd_ngram* const* ctxs, const int32_t* prompts,
+                                int prompt_len, int max_new, int K, int32_t* out, anpd_stats* stats) {
+    return generate_core(m, kv, ctxs, prompts, prompt_len, max_new, K, out, stats, false);
+}
+
 anpd_status anpd_generate(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const int32_t* prompt, int prompt_len,
                           int max_new, int K, int32_t* out, int* n_out, anpd_stats* stats) {
     if (!kv || kv->batch != 1 || !n_out) return ANPD_ERR_ARG;
     anpd_ngram* arr[1] = {ctx};
-    ANPD_TRY(anpd_generate_batch(m, kv, arr, prompt, prompt_len, max_new, K, out, stats));
+    ANPD_TRY(generate_core(m, kv, arr, prompt, prompt_len, max_new, K, out, stats, false));
     *n_out = max_new;
     return ANPD_OK;
+}
+
+anpd_status anpd_generate_dev(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const int32_t* prompt_dev, int prompt_len,
+                              int max_new, int K, int32_t* out_dev, int* n_out, anpd_stats* stats) {
+    if (!kv || kv->batch != 1 || !n_out) return ANPD_ERR_ARG;
+    anpd_ngram* arr[1] = {ctx};
+    ANPD_TRY(generate_core(m, kv, arr, prompt_dev, prompt_len, max_new, K, out_dev, stats, true));
+    *n_out = max_new;
+    return ANPD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// GEMM test hook
+// ---------------------------------------------------------------------------------------------
+anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a, int rows, float* out, int plain) {
+    if (!w_bf16 || !a || !out || N < 1 || K < 8 || K % 8 || rows < 8 || rows % 8 || rows > 128) return ANPD_ERR_ARG;
+    if (!have_device()) return ANPD_ERR_CUDA;
+    int dev = 0, sms = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    GemmPlan plan;
+    gemm_make_plan(&plan, N, K, sms);
+    const int NB = (rows + 15) / 16 * 16;
+    const int segs = plain ? 1 : plan.max_segs;
+    std::vector<uint16_t> hi((size_t)rows * K), lo((size_t)rows * K);
+    for (size_t i = 0; i < hi.size(); ++i) {
+        hi[i] = f32_to_bf16_host(a[i]);
+        uint32_t u = (uint32_t)hi[i] << 16;
+        float h; std::memcpy(&h, &u, 4);
+        lo[i] = f32_to_bf16_host(a[i] - h);
+    }
+    const size_t wb = up256((size_t)N * K * 2), ab = up256((size_t)rows * K * 2), pb = up256((size_t)segs * rows * N * 4),
+                 tb = up256((size_t)plan.m_tiles * 4);
+    char* slab = nullptr;
+    if (cudaMalloc((void**)&slab, wb + 2 * ab + pb + tb + 256) != cudaSuccess) { cudaGetLastError(); return ANPD_ERR_OOM; }
+    bf16* dW = (bf16*)slab; bf16* dhi = (bf16*)(slab + wb); bf16* dlo = (bf16*)(slab + wb + ab);
+    float* dpart = (float*)(slab + wb + 2 * ab);
+    int* dfirst = (int*)(slab + wb + 2 * ab + pb);
+    int* derr = (int*)(slab + wb + 2 * ab + pb + tb);
+    plan.d_first_cta = dfirst;
+    anpd_status rc = ANPD_OK;
+    auto body = [&]() -> anpd_status {
+        CUDA_TRY(cudaMemset(slab + wb + 2 * ab, 0, pb + tb + 256));
+        CUDA_TRY(cudaMemcpy(dW, w_bf16, (size_t)N * K * 2, cudaMemcpyHostToDevice));
+        CUDA_TRY(cudaMemcpy(dhi, hi.data(), hi.size() * 2, cudaMemcpyHostToDevice));
+        CUDA_TRY(cudaMemcpy(dlo, lo.data(), lo.size() * 2, cudaMemcpyHostToDevice));
+        CUDA_TRY(cudaMemcpy(dfirst, plan.first_cta.data(), (size_t)plan.m_tiles * 4, cudaMemcpyHostToDevice));
+        if (plain) {
+            ANPD_TRY(gemm_plain_enqueue(dW, dhi, dlo, rows, N, K, dpart, N, 0, nullptr));
+        } else {
+            CUtensorMap mw, mh, ml;
+            ANPD_TRY(make_tmap_bf16(&mw, dW, N, K, 128, true));
+            ANPD_TRY(make_tmap_bf16(&mh, dhi, rows, K, NB, false));
+            ANPD_TRY(make_tmap_bf16(&ml, dlo, rows, K, NB, false));
+            ANPD_TRY(gemm_tc_enqueue(plan, mw, mh, ml, rows, NB, dpart, (size_t)rows * N, N, derr, 0, nullptr));
+        }
+        CUDA_TRY(cudaDeviceSynchronize());
+        int err = 0;
+        CUDA_TRY(cudaMemcpy(&err, derr, 4, cudaMemcpyDeviceToHost));
+        if (err) { std::snprintf(g_last_error, sizeof(g_last_error), "GEMM kernel gave up waiting (code %d)", err); return ANPD_ERR_CUDA; }
+        std::vector<float> part((size_t)segs * rows * N);
+        CUDA_TRY(cudaMemcpy(part.data(), dpart, part.size() * 4, cudaMemcpyDeviceToHost));
+        for (int r = 0; r < rows; ++r)
+            for (int n = 0; n < N; ++n) {
+                const int ns = plain ? 1 : plan.seg_count[n >> 7];
+                float acc = 0.0f;
+                for (int sgm = 0; sgm < ns; ++sgm) acc += part[((size_t)sgm * rows + r) * N + n];
+                out[(size_t)r * N + n] = acc;
+            }
+        return ANPD_OK;
+    };
+    rc = body();
+    cudaFree(slab);
+    return rc;
 }
 
 // ---------------------------------------------------------------------------------------------

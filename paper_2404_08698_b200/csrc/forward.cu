@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const bf16* __restrict_
 }
 
 // x[row] += sum over splits of part[s][row]; then h = rmsnorm(x) * gain, split into hi + lo.
-__global__ void __launch_bounds__(256) resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, int splits,
+__global__ void __launch_bounds__(256) resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, const int* __restrict__ seg_count,
                                                          size_t split_stride, int ld_part, const float* __restrict__ gain,
                                                          float eps, int d, bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
     __shared__ float red[8];
@@ -102,7 +102,8 @@ __global__ void __launch_bounds__(256) resid_norm_kernel(float* __restrict__ x, 
     float ss = 0.0f;
     for (int i = threadIdx.x; i < d; i += 256) {
         float v = xr[i];
-        for (int s = 0; s < splits; ++s) v += part[s * split_stride + (size_t)row * ld_part + i];
+        const int ns = seg_count[i >> 7];
+        for (int s = 0; s < ns; ++s) v += part[s * split_stride + (size_t)row * ld_part + i];
         xr[i] = v;
         ss += v * v;
     }
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(256) resid_norm_kernel(float* __restrict__ x, 
 // ---------------------------------------------------------------------------------------------
 // QKV epilogue: reduce splits, rotary embedding, append K/V to the paged cache, keep q
 // ---------------------------------------------------------------------------------------------
-__global__ void qkv_rope_append_kernel(const float* __restrict__ part, int splits, size_t split_stride, int ld_part,
+__global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride, int ld_part,
                                        const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                                        const int* __restrict__ row_ok, const float* __restrict__ rope_cos,
                                        const float* __restrict__ rope_sin, const int* __restrict__ page_table,
@@ -127,7 +128,8 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, int split
     const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
     const float* pr = part + (size_t)row * ld_part + (size_t)head * hd;
     float a = 0.0f, b = 0.0f;
-    for (int s = 0; s < splits; ++s) { a += pr[s * split_stride + i]; b += pr[s * split_stride + i + half]; }
+    const int ns = seg_count[(head * hd + i) >> 7];      // a head never straddles a 128-column tile
+    for (int s = 0; s < ns; ++s) { a += pr[s * split_stride + i]; b += pr[s * split_stride + i + half]; }
     const int pos = row_pos[row];
     if (head < Hq + Hkv) {
         const float c = rope_cos[(size_t)pos * half + i], sn = rope_sin[(size_t)pos * half + i];
@@ -294,13 +296,15 @@ __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* _
 // ---------------------------------------------------------------------------------------------
 // SwiGLU epilogue of the gate/up projection
 // ---------------------------------------------------------------------------------------------
-__global__ void swiglu_kernel(const float* __restrict__ part, int splits, size_t split_stride, int ld_part, int F,
+__global__ void swiglu_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride, int ld_part, int F,
                               bf16* __restrict__ act_hi, bf16* __restrict__ act_lo) {
     const int row = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= F) return;
     const float* pr = part + (size_t)row * ld_part;
     float gte = 0.0f, up = 0.0f;
-    for (int s = 0; s < splits; ++s) { gte += pr[s * split_stride + j]; up += pr[s * split_stride + F + j]; }
+    const int ng = seg_count[j >> 7], nu = seg_count[(F + j) >> 7];
+    for (int s = 0; s < ng; ++s) gte += pr[s * split_stride + j];
+    for (int s = 0; s < nu; ++s) up += pr[s * split_stride + F + j];
     const float v = gte / (1.0f + expf(-gte)) * up;
     bf16 hi, lo;
     split_bf16(v, hi, lo);
@@ -312,7 +316,7 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int splits, size_t
 // LM-head epilogue: reduce splits, (optionally) keep logits, per-block argmax with ties to the lowest id
 // ---------------------------------------------------------------------------------------------
 constexpr int AMAX_COLS = 1024;
-__global__ void __launch_bounds__(256) argmax_partial_kernel(const float* __restrict__ part, int splits, size_t split_stride,
+__global__ void __launch_bounds__(256) argmax_partial_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride,
                                                              int ld_part, int V, float* __restrict__ logits,
                                                              float* __restrict__ amax_val, int* __restrict__ amax_idx, int nblk) {
     __shared__ float sv[8];
@@ -325,7 +329,8 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const float* __rest
         const int v = blockIdx.x * AMAX_COLS + u * 256 + threadIdx.x;
         if (v < V) {
             float z = 0.0f;
-            for (int s = 0; s < splits; ++s) z += pr[s * split_stride + v];
+            const int ns = seg_count[v >> 7];
+            for (int s = 0; s < ns; ++s) z += pr[s * split_stride + v];
             if (logits) logits[(size_t)row * V + v] = z;
             if (z > best) { best = z; bidx = v; }       // ascending v: strict > keeps the lowest id
         }
@@ -449,12 +454,25 @@ __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict_
     }
 }
 
-anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, const bf16* W, const bf16* a_hi, const bf16* a_lo, int rows,
-                         int N, int K, int* splits_out) {
+// One projection of the forward.  Returns the per-tile segment counts its consumer must use.
+anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int rows, const int** seg_count_out) {
     Workspace& ws = kv->ws;
-    LAUNCH(&m->prof, m->stream, KC_GEMM, 2.0 * (double)N * (double)K,
-           (gemm_rows8_kernel<<<(N + 7) / 8, 256, 0, m->stream>>>(W, a_hi, a_lo, rows, N, K, ws.part, ws.n_max_out)));
-    *splits_out = 1;
+    const GemmPlan& plan = m->plan[kind];
+    const int mode = (rows == kv->batch * ANPD_ROWS) ? 0 : 1;
+    const bf16* W = kind == GK_LM ? m->lm_head : (kind == GK_QKV ? m->layers[layer].wqkv : kind == GK_O ? m->layers[layer].wo
+                                                 : kind == GK_GU ? m->layers[layer].wgu : m->layers[layer].wd);
+    const bf16 *a_hi = ws.h_hi, *a_lo = ws.h_lo;
+    const CUtensorMap* maps = ws.map_h[mode];
+    if (kind == GK_O) { a_hi = ws.ao_hi; a_lo = ws.ao_lo; maps = ws.map_ao[mode]; }
+    if (kind == GK_DOWN) { a_hi = ws.act_hi; a_lo = ws.act_lo; maps = ws.map_act[mode]; }
+    if (m->plain_gemm) {
+        *seg_count_out = m->d_ones;
+        return gemm_plain_enqueue(W, a_hi, a_lo, rows, plan.N, plan.K, ws.part, ws.n_max_out, m->stream, &m->prof);
+    }
+    const CUtensorMap& mw = kind == GK_LM ? m->map_lm : m->layers[layer].map[kind];
+    ANPD_TRY(gemm_tc_enqueue(plan, mw, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)ws.r_max * ws.n_max_out,
+                             ws.n_max_out, ws.gemm_err, m->stream, &m->prof));
+    *seg_count_out = plan.d_seg_count;
     return ANPD_OK;
 }
 
@@ -484,6 +502,14 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
 }
 
 }  // namespace
+
+anpd_status gemm_plain_enqueue(const bf16* W, const bf16* a_hi, const bf16* a_lo, int rows, int N, int K, float* part, int ld_part,
+                               cudaStream_t st, Profiler* prof) {
+    LAUNCH(prof, st, KC_GEMM, 2.0 * (double)N * (double)K,
+           (gemm_rows8_kernel<<<(N + 7) / 8, 256, 0, st>>>(W, a_hi, a_lo, rows, N, K, part, ld_part)));
+    CUDA_TRY(cudaGetLastError());
+    return ANPD_OK;
+}
 
 anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv) {
     Workspace& ws = kv->ws;
@@ -522,38 +548,38 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     const int d = c.d_model, F = c.d_ffn, hd = c.head_dim, V = c.vocab;
     const size_t sstride = (size_t)ws.r_max * ws.n_max_out;
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * hd;
-    int splits = 1;
+    const int* segs = nullptr;
 
     LAUNCH(pf, st, KC_OTHER, 0, (embed_norm_kernel<<<rows, 256, 0, st>>>(m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
                                                                       ws.x, ws.h_hi, ws.h_lo)));
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& w = m->layers[l];
-        ANPD_TRY(gemm_enqueue(m, kv, w.wqkv, ws.h_hi, ws.h_lo, rows, m->nqkv, d, &splits));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_QKV, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
                (qkv_rope_append_kernel<<<dim3(rows, c.n_q_heads + 2 * c.n_kv_heads), hd / 2, 0, st>>>(
-                   ws.part, splits, sstride, ws.n_max_out, ws.row_pos, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
+                   ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
                    kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, hd, ws.q, kv->kpool + l * layer_elems,
                    kv->vpool + l * layer_elems)));
         if (hd == 128) ANPD_TRY(attn_enqueue<128>(m, kv, l, rows, max_pos));
         else ANPD_TRY(attn_enqueue<64>(m, kv, l, rows, max_pos));
-        ANPD_TRY(gemm_enqueue(m, kv, w.wo, ws.ao_hi, ws.ao_lo, rows, d, m->dq, &splits));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_O, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (resid_norm_kernel<<<rows, 256, 0, st>>>(ws.x, ws.part, splits, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
+               (resid_norm_kernel<<<rows, 256, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
-        ANPD_TRY(gemm_enqueue(m, kv, w.wgu, ws.h_hi, ws.h_lo, rows, 2 * F, d, &splits));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (swiglu_kernel<<<dim3((F + 255) / 256, rows), 256, 0, st>>>(ws.part, splits, sstride, ws.n_max_out, F, ws.act_hi,
+               (swiglu_kernel<<<dim3((F + 255) / 256, rows), 256, 0, st>>>(ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
                                                                           ws.act_lo)));
-        ANPD_TRY(gemm_enqueue(m, kv, w.wd, ws.act_hi, ws.act_lo, rows, d, F, &splits));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_DOWN, l, rows, &segs));
         const float* next_gain = (l + 1 < c.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
         LAUNCH(pf, st, KC_OTHER, 0,
-               (resid_norm_kernel<<<rows, 256, 0, st>>>(ws.x, ws.part, splits, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
+               (resid_norm_kernel<<<rows, 256, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
     }
     if (!head) { CUDA_TRY(cudaGetLastError()); return ANPD_OK; }
-    ANPD_TRY(gemm_enqueue(m, kv, m->lm_head, ws.h_hi, ws.h_lo, rows, V, d, &splits));
+    ANPD_TRY(gemm_enqueue(m, kv, GK_LM, 0, rows, &segs));
     LAUNCH(pf, st, KC_OTHER, 0,
-           (argmax_partial_kernel<<<dim3(ws.amax_blocks, rows), 256, 0, st>>>(ws.part, splits, sstride, ws.n_max_out, V,
+           (argmax_partial_kernel<<<dim3(ws.amax_blocks, rows), 256, 0, st>>>(ws.part, segs, sstride, ws.n_max_out, V,
                                                                              want_logits ? ws.logits : nullptr, ws.amax_val,
                                                                              ws.amax_idx, ws.amax_blocks)));
     CUDA_TRY(cudaGetLastError());

@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units (not part of the boundary).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -128,6 +129,17 @@ anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batc
 constexpr int KV_PAGE = 128;          // positions per KV page (= key chunk of one attention block)
 constexpr int PREFILL_ROWS = 64;      // rows per prefill pass
 
+// How one [N][K] weight matrix is cut across the persistent GEMM CTAs (depends on the shape and the
+// SM count only): tile t is started by CTA first_cta[t] and covered by seg_count[t] consecutive CTAs,
+// each of which leaves one partial sum; consumers add them in that order.
+struct GemmPlan {
+    int N, K, m_tiles, k_blocks, grid, max_segs;
+    std::vector<int> first_cta, seg_count;
+    int* d_first_cta;
+    int* d_seg_count;
+};
+enum GemmKind { GK_QKV = 0, GK_O = 1, GK_GU = 2, GK_DOWN = 3, GK_LM = 4, GK_COUNT = 5 };
+
 struct LayerW {
     const __nv_bfloat16* wqkv;        // [(Hq + 2 Hkv) * hd, d]  (q rows, then k rows, then v rows)
     const __nv_bfloat16* wo;          // [d, Hq * hd]
@@ -135,6 +147,7 @@ struct LayerW {
     const __nv_bfloat16* wd;          // [d, F]
     const float* attn_norm;           // [d]
     const float* ffn_norm;            // [d]
+    CUtensorMap map[4];               // TMA views of wqkv, wo, wgu, wd (128-row x 64-column boxes)
 };
 
 struct anpd_model {
@@ -148,6 +161,13 @@ struct anpd_model {
     void* slab;
     size_t slab_bytes;
     double streamed_bytes;            // weight bytes one forward reads
+    CUtensorMap map_lm;
+    GemmPlan plan[GK_COUNT];
+    int* d_plan_tables;               // device copies of the plans' tables
+    int* d_ones;                      // [tiles] all 1: segment counts of the plain GEMM
+    int max_segs;
+    bool plain_gemm;                  // debugging aid: route GEMMs through the plain kernel
+    int num_sms;
     Profiler prof;
 };
 
@@ -166,6 +186,10 @@ struct Workspace {
     float* logits;                    // [r_max, V]
     float* amax_val; int* amax_idx;   // [r_max, amax_blocks]
     int amax_blocks;
+    int* gemm_err;                    // device flag set by a GEMM kernel that gave up waiting
+    // TMA views of the activation buffers: [0] decode (batch*8 rows), [1] prefill (PREFILL_ROWS rows)
+    CUtensorMap map_h[2][2], map_ao[2][2], map_act[2][2];     // [mode][hi/lo]
+    int nb[2];                        // MMA N per mode (rows padded to a multiple of 16)
 };
 
 struct anpd_kv {
@@ -199,3 +223,13 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
 // `seq` gives the first generated token, kv_len becomes prompt_len.  d_ctxs may be null; otherwise
 // accepted tokens and the next token are appended to the sequences' token buffers.
 anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len);
+
+// gemm_tc.cu
+anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, int box_rows, bool streamed);
+void gemm_make_plan(GemmPlan* p, int N, int K, int num_sms);
+anpd_status gemm_tc_enqueue(const GemmPlan& plan, const CUtensorMap& map_w, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
+                            int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,
+                            Profiler* prof);
+// forward.cu: the plain (one warp per output feature) GEMM, kept as a cross-check
+anpd_status gemm_plain_enqueue(const __nv_bfloat16* W, const __nv_bfloat16* a_hi, const __nv_bfloat16* a_lo, int rows, int N, int K,
+                               float* part, int ld_part, cudaStream_t st, Profiler* prof);

@@ -30,27 +30,20 @@ def top2_margin(logits_row: torch.Tensor) -> float:
     return float(t[0] - t[1])
 
 
-def oracle_greedy_with_margins(dec, prompt, max_new):
-    """Oracle greedy tokens and, per generated token, the top-2 logit margin that decided it."""
+def check_stream_against_oracle(dec, prompt, got, min_margin=5e-2) -> int:
+    """Teacher-forced comparison of a generated token stream with the oracle: the oracle
+    consumes the prompt and then the stream itself, and at every position whose top-2 logit
+    margin exceeds min_margin its argmax must be the stream's token (below the margin a
+    rounding difference may legitimately pick the other candidate).  Returns the number of
+    positions that were decided by a large enough margin."""
     from oracle.anpd import argmax_lowest
     cache = dec.new_cache()
     logits = dec.forward(list(prompt), cache)
-    toks, margins = [argmax_lowest(logits[-1])], [top2_margin(logits[-1])]
-    while len(toks) < max_new:
-        logits = dec.forward([toks[-1]], cache)
-        toks.append(argmax_lowest(logits[-1]))
-        margins.append(top2_margin(logits[-1]))
-    return toks, margins
-
-
-def agree_until_low_margin(got, want, margins, min_margin=5e-2) -> int:
-    """Asserts got[i] == want[i] up to the first position whose deciding margin is below
-    min_margin (beyond it a rounding difference may legitimately change the stream).
-    Returns the number of positions checked."""
-    n = 0
-    for g, w, mg in zip(got, want, margins):
-        if mg <= min_margin:
-            break
-        assert int(g) == int(w), f"token {n}: got {g}, oracle {w}, margin {mg}"
-        n += 1
-    return n
+    checked = 0
+    for i, tok in enumerate(got):
+        if top2_margin(logits[-1]) > min_margin:
+            want = argmax_lowest(logits[-1])
+            assert int(tok) == want, f"token {i}: got {int(tok)}, oracle {want}, margin {top2_margin(logits[-1])}"
+            checked += 1
+        logits = dec.forward([int(tok)], cache)
+    return checked

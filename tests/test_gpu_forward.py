@@ -78,8 +78,8 @@ def test_verify_decisions_match_oracle(A, c1):
     c1.dec_bf16.forward(prompt, cache)
     rng = np.random.default_rng(0)
     checked = 0
-    for step in range(12):
-        # build a draft that follows the oracle's own predictions for a random number of tokens
+    for step in range(40):
+        # a draft that follows the oracle's own predictions for `good` tokens, then departs
         P = cache.length
         k = int(rng.integers(0, 8))
         good = int(rng.integers(0, k + 1))
@@ -97,15 +97,14 @@ def test_verify_decisions_match_oracle(A, c1):
         a_want = accept_length(draft, preds)
         safe = all(top2_margin(logits[r]) > MARGIN for r in range(a_want + 1))
         a, nxt = A.anpd_verify(c1.m, c1.kv, last, draft)
-        if not safe:
-            break
-        assert (a, nxt) == (a_want, preds[a_want]), (step, draft, preds)
-        assert a >= min(good, k)
-        assert A.anpd_kv_len(c1.kv) == P + a + 1
+        assert 0 <= a <= k and A.anpd_kv_len(c1.kv) == P + a + 1
+        if safe:
+            assert (a, nxt) == (a_want, preds[a_want]), (step, draft, preds)
+            checked += 1
+        # follow the library's decision so both sides stay on one stream
         cache.truncate(P + a + 1)
         last = nxt
-        checked += 1
-    assert checked >= 3
+    assert checked >= 5, checked
 
 
 def test_rows_are_independent_of_row_count_and_drafts(A, c1):

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import agree_until_low_margin, as_bf16_values, gpu_model, oracle_greedy_with_margins, require_gpu
+from helpers import as_bf16_values, check_stream_against_oracle, gpu_model, require_gpu
 from oracle.anpd import anpd_generate as oracle_anpd
 from oracle.decoder import Decoder
 from oracle.mln import MLN
@@ -46,12 +46,12 @@ def test_c1_anpd_equals_greedy_equals_oracle(A, c1):
         assert sum(st["hist_accepted"]) == st["steps"] and sum(st["hist_accepted"][wl.K + 1:]) == 0
         assert st["accepted"] == sum(i * h for i, h in enumerate(st["hist_accepted"]))
         dec = Decoder(wl.shape, as_bf16_values(w), torch.float64)
-        want, margins = oracle_greedy_with_margins(dec, prompt.tolist(), wl.max_new)
-        n = agree_until_low_margin(ref, want, margins)
-        assert n >= 8, n
-        if n == wl.max_new:
-            # same stream: the oracle's Algorithm 1 must have taken the same steps
-            _, ost, _ = oracle_anpd(dec, prompt.tolist(), wl.max_new, wl.K, n_max=wl.n_max)
+        n = check_stream_against_oracle(dec, prompt.tolist(), ref.tolist())
+        assert n >= wl.max_new // 5, n
+        # the oracle's Algorithm 1 on the same stream: if its own greedy stream is the library's,
+        # it must have taken the same steps (same drafts, same accepted lengths)
+        want, ost, _ = oracle_anpd(dec, prompt.tolist(), wl.max_new, wl.K, n_max=wl.n_max)
+        if want == ref.tolist():
             assert st["steps"] == ost.steps and st["accepted"] == ost.accepted and st["drafted"] == ost.drafted
             assert st["hist_accepted"] == ost.hist_accepted
     finally:
@@ -67,10 +67,12 @@ def test_tables_after_generate_match_oracle_on_the_generated_stream(A, c1):
         out, st = A.anpd_generate(m, kv, ctx, prompt, 40, 5)
         assert np.array_equal(out, ref[:40])
         n_ctx = A.anpd_ngram_len(ctx)
-        assert n_ctx == len(prompt) + st["generated"] and 40 <= st["generated"] <= 45
+        # the context also holds the token confirmed by the last step, which Algorithm 1 would
+        # only move to the output at the top of its next iteration
+        assert n_ctx == len(prompt) + st["generated"] + 1 and 40 <= st["generated"] <= 45
         assert A.anpd_kv_len(kv) == n_ctx - 1                           # the last token is not in the cache yet
         # the loop may overshoot max_new; by losslessness the context holds the greedy stream
-        committed = prompt.tolist() + ref[:st["generated"]].tolist()
+        committed = prompt.tolist() + ref[:st["generated"] + 1].tolist()
         assert A.anpd_ngram_draft(ctx, 0) == []                         # folds the last step's tokens
         mln = MLN(2, 4)
         mln.initialize(committed)
