@@ -145,6 +145,62 @@ def run_reference(args) -> None:
     }))
 
 
+def verify_microbench(args, A, wl, model, stream) -> None:
+    """The verify step alone (workload C4): for each KV length, verify width K+1 and forced acceptance
+    probability p, drafts are built left to right from the model's own argmax (draft_i = the model's
+    token with probability p, else a different token), then the step is timed with CUDA events."""
+    from workloads import markov_prompt
+    from workloads.rng import uniform_at
+    shape = wl.shape
+    peak, peak_kind = measured_hbm_peak()
+    rows_out = []
+    for kv_len in args.kv_len:
+        kv = A.anpd_kv_create(model, kv_len + 64)
+        prompt = markov_prompt(kv_len, shape.vocab, wl.markov_order, wl.prompt_seed + 17, copy_spans=wl.copy_spans)
+        first = A.anpd_prefill(model, kv, prompt)
+        P = A.anpd_kv_len(kv)
+        for width in args.widths:
+            k = width - 1
+            for p in (args.accept_p if k > 0 else [0.0]):
+                times, hist = [], [0] * 8
+                for ds in range(args.draft_sets if k > 0 else 1):
+                    draft = []
+                    for i in range(k):                      # untimed dry runs, one per draft position
+                        logits = A.anpd_verify_logits(model, kv, first, draft, shape.vocab)
+                        pred = int(np.argmax(logits[i]))
+                        keep = uniform_at(977 + ds, width * 16 + int(p * 100), i) < p
+                        draft.append(pred if keep else (pred + 1) % shape.vocab)
+                    A.anpd_verify_stage(model, kv, [first], [draft])
+                    for _ in range(3):
+                        A.anpd_verify_enqueue(model, kv)
+                        A.anpd_kv_truncate(kv, 0, P)
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    for _ in range(args.verify_iters):
+                        A.anpd_verify_enqueue(model, kv)
+                        A.anpd_kv_truncate(kv, 0, P)
+                    e1.record(stream)
+                    torch.cuda.synchronize()
+                    times.append(e0.elapsed_time(e1) / args.verify_iters)
+                    acc, _ = A.anpd_verify_result(model, kv)
+                    A.anpd_kv_truncate(kv, 0, P)
+                    hist[acc[0]] += 1
+                ms = statistics.median(times)
+                nbytes = shape.streamed_params * 2 + shape.kv_bytes_per_token * (P + A.ROWS)
+                gbs = nbytes / (ms * 1e-3) / 1e9
+                mean_acc = sum(i * h for i, h in enumerate(hist)) / max(sum(hist), 1)
+                rows_out.append({"kv_len": P, "width": width, "p": p, "ms": ms, "gbs": gbs, "frac_of_8TBs": gbs / HBM_NOMINAL_GBS,
+                                 f"frac_of_{peak_kind}_copy": gbs / peak, "accepted_hist": hist,
+                                 "tokens_per_s_at_this_acceptance": (1 + mean_acc) / (ms * 1e-3)})
+        A.anpd_kv_destroy(kv)
+    best = min(r["ms"] for r in rows_out)
+    print(json.dumps({"metric": "verify_step_ms", "value": best, "unit": "ms", "higher_is_better": False, "n_gpus": 1,
+                      "dtype": "bf16", "data": "synthetic", "launches": A.anpd_launch_count(),
+                      "config": {"workload": f"C4 verify-step microbenchmark on the {wl.name} model", "iters": args.verify_iters},
+                      "rows": rows_out}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -154,6 +210,12 @@ def main() -> None:
     ap.add_argument("--workload", default="C3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--verify-iters", type=int, default=40)
+    ap.add_argument("--mode", default="generate", choices=["generate", "verify"],
+                    help="verify: the verify-step microbenchmark only (KV length, widths, forced acceptance)")
+    ap.add_argument("--kv-len", type=int, nargs="+", default=[2048, 4096])
+    ap.add_argument("--widths", type=int, nargs="+", default=[1, 2, 4, 6, 8])
+    ap.add_argument("--accept-p", type=float, nargs="+", default=[0.0, 0.5, 0.9])
+    ap.add_argument("--draft-sets", type=int, default=4)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -185,6 +247,10 @@ def main() -> None:
     w_cpu = {k: v.cpu() for k, v in w.items()} if want_cpu else None
     del w
     torch.cuda.empty_cache()
+    if args.mode == "verify":
+        verify_microbench(args, A, wl, model, stream)
+        A.anpd_model_destroy(model)
+        return
     max_len = wl.prompt_len + wl.max_new + 64
     kv = A.anpd_kv_create(model, max_len)
     ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, stream.cuda_stream)

@@ -58,7 +58,7 @@ typedef struct anpd_ngram anpd_ngram; /* one sequence's token buffer + MLN table
  * embedding with pairs (i, i + head_dim/2) and angle pos * theta^(-2i/head_dim), grouped-query
  * attention with softmax scale 1/sqrt(head_dim), SwiGLU FFN, no biases, untied LM head.
  * Requirements: d_model, d_ffn and n_q_heads*head_dim multiples of 8; head_dim 64 or 128;
- * n_q_heads a multiple of n_kv_heads with at most 8 query heads per kv head. */
+ * 1, 2, 4 or 8 query heads per kv head; d_model <= 16384. */
 typedef struct {
     int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
     float rope_theta, rms_eps;

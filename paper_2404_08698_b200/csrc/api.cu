@@ -141,12 +141,12 @@ static anpd_status model_make_plans(anpd_model* m) {
     CUDA_TRY(cudaMemcpy(m->d_plan_tables, host.data(), ints * sizeof(int), cudaMemcpyHostToDevice));
     for (int l = 0; l < c.n_layers; ++l) {
         LayerW& w = m->layers[l];
-        ANPD_TRY(make_tmap_bf16(&w.map[GK_QKV], w.wqkv, m->nqkv, c.d_model, 128, true));
-        ANPD_TRY(make_tmap_bf16(&w.map[GK_O], w.wo, c.d_model, m->dq, 128, true));
-        ANPD_TRY(make_tmap_bf16(&w.map[GK_GU], w.wgu, 2 * c.d_ffn, c.d_model, 128, true));
-        ANPD_TRY(make_tmap_bf16(&w.map[GK_DOWN], w.wd, c.d_model, c.d_ffn, 128, true));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_QKV], w.wqkv, m->nqkv, c.d_model));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_O], w.wo, c.d_model, m->dq));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_GU], w.wgu, 2 * c.d_ffn, c.d_model));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_DOWN], w.wd, c.d_model, c.d_ffn));
     }
-    ANPD_TRY(make_tmap_bf16(&m->map_lm, m->lm_head, c.vocab, c.d_model, 128, true));
+    ANPD_TRY(make_tmap_tiled(&m->map_lm, m->lm_head, c.vocab, c.d_model));
     return ANPD_OK;
 }
 
@@ -180,7 +180,11 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     const anpd_model_config& c = *cfg;
     if (c.n_layers < 1 || c.d_model < 8 || c.n_q_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 8 || c.vocab < 1) return ANPD_ERR_ARG;
     if (c.head_dim != 64 && c.head_dim != 128) return ANPD_ERR_ARG;
-    if (c.n_q_heads % c.n_kv_heads != 0 || c.n_q_heads / c.n_kv_heads > 8) return ANPD_ERR_ARG;
+    {
+        const int grp = c.n_q_heads / c.n_kv_heads;          // query heads per kv head
+        if (c.n_q_heads % c.n_kv_heads != 0 || (grp != 1 && grp != 2 && grp != 4 && grp != 8)) return ANPD_ERR_ARG;
+    }
+    if (c.d_model > 16384) return ANPD_ERR_ARG;
     if (c.d_model % 8 || c.d_ffn % 8 || c.vocab >= (1 << 24)) return ANPD_ERR_ARG;
     if (!(c.rope_theta > 0.0f) || !(c.rms_eps >= 0.0f)) return ANPD_ERR_ARG;
     const int n_tensors = 1 + 9 * c.n_layers + 2;
@@ -195,9 +199,14 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     m->dkv = c.n_kv_heads * c.head_dim;
     m->nqkv = m->dq + 2 * m->dkv;
     const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
-    const size_t b_embed = up256(V * d * 2), b_qkv = up256((size_t)m->nqkv * d * 2), b_o = up256(d * m->dq * 2),
-                 b_gu = up256(2 * F * d * 2), b_d = up256(d * F * 2), b_norm = up256(d * 4);
-    m->slab_bytes = 2 * b_embed + b_norm + c.n_layers * (b_qkv + b_o + b_gu + b_d + 2 * b_norm);
+    // GEMM weights are stored tile by tile (128 output rows x 64 inputs, 16 KB contiguous each, zero
+    // padded at ragged edges) so that every TMA box is one contiguous read; the embedding table stays
+    // row-major because it is only gathered.
+    const size_t b_embed = up256(V * d * 2), b_lm = up256(gemm_tiled_elems((int)V, (int)d) * 2),
+                 b_qkv = up256(gemm_tiled_elems(m->nqkv, (int)d) * 2), b_o = up256(gemm_tiled_elems((int)d, m->dq) * 2),
+                 b_gu = up256(gemm_tiled_elems(2 * (int)F, (int)d) * 2), b_d = up256(gemm_tiled_elems((int)d, (int)F) * 2),
+                 b_norm = up256(d * 4);
+    m->slab_bytes = b_embed + b_lm + b_norm + c.n_layers * (b_qkv + b_o + b_gu + b_d + 2 * b_norm);
     if (cudaMalloc(&m->slab, m->slab_bytes) != cudaSuccess) { cudaGetLastError(); delete m; return ANPD_ERR_OOM; }
     m->streamed_bytes = 2.0 * ((double)c.n_layers * ((double)m->nqkv * d + (double)d * m->dq + 3.0 * F * d) + (double)V * d);
 
@@ -206,11 +215,28 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     const bool bf = weights_are_bf16 != 0, dev = weights_on_device != 0;
     cudaStream_t st = m->stream;
     anpd_status rc = ANPD_OK;
+    // staging for host-side sources: the largest matrix in its source type
+    void* stage = nullptr;
+    const size_t max_elems = std::max(std::max((size_t)V * d, F * d), std::max((size_t)m->dq * d, d * F));
+    if (!dev && cudaMalloc(&stage, max_elems * (bf ? 2 : 4)) != cudaSuccess) { cudaGetLastError(); cudaFree(m->slab); delete m; return ANPD_ERR_OOM; }
+    if (cudaMemsetAsync(m->slab, 0, m->slab_bytes, st) != cudaSuccess) rc = ANPD_ERR_CUDA;
     auto put = [&](const void* src, size_t n, bool as_bf16, size_t bytes) -> void* {
         void* dst = p;
         p += bytes;
         if (rc == ANPD_OK) rc = upload(dst, src, n, as_bf16, bf, dev, st, tmp, nullptr, 0);
         return dst;
+    };
+    // rows [row_off, row_off + rows) of a tiled [*, K] matrix at dst
+    auto put_tiled = [&](const void* src, int rows, int K, int row_off, void* dst) {
+        if (rc != ANPD_OK) return;
+        const void* dsrc = src;
+        if (!dev) {
+            if (cudaMemcpyAsync(stage, src, (size_t)rows * K * (bf ? 2 : 4), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+                cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; return; }
+            dsrc = stage;
+        }
+        rc = gemm_retile_enqueue(dsrc, !bf, rows, K, row_off, (bf16*)dst, st);
+        if (rc == ANPD_OK && !dev && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
     };
     int t = 0;
     m->embed = (const bf16*)put(weights[t++], V * d, true, b_embed);
@@ -218,25 +244,30 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     for (int l = 0; l < c.n_layers; ++l) {
         LayerW& w = m->layers[l];
         w.attn_norm = (const float*)put(weights[t++], d, false, b_norm);
-        // q, k and v rows are stored back to back so that one GEMM produces all three
-        char* qkv = p;
-        put(weights[t++], (size_t)m->dq * d, true, (size_t)m->dq * d * 2);
-        put(weights[t++], (size_t)m->dkv * d, true, (size_t)m->dkv * d * 2);
-        put(weights[t++], (size_t)m->dkv * d, true, (size_t)m->dkv * d * 2);
-        p = qkv + b_qkv;
-        w.wqkv = (const bf16*)qkv;
-        w.wo = (const bf16*)put(weights[t++], d * m->dq, true, b_o);
+        // q, k and v rows form one matrix so that one GEMM produces all three
+        w.wqkv = (const bf16*)p;
+        put_tiled(weights[t++], m->dq, (int)d, 0, p);
+        put_tiled(weights[t++], m->dkv, (int)d, m->dq, p);
+        put_tiled(weights[t++], m->dkv, (int)d, m->dq + m->dkv, p);
+        p += b_qkv;
+        w.wo = (const bf16*)p;
+        put_tiled(weights[t++], (int)d, m->dq, 0, p);
+        p += b_o;
         w.ffn_norm = (const float*)put(weights[t++], d, false, b_norm);
-        char* gu = p;
-        put(weights[t++], F * d, true, F * d * 2);
-        put(weights[t++], F * d, true, F * d * 2);
-        p = gu + b_gu;
-        w.wgu = (const bf16*)gu;
-        w.wd = (const bf16*)put(weights[t++], d * F, true, b_d);
+        w.wgu = (const bf16*)p;
+        put_tiled(weights[t++], (int)F, (int)d, 0, p);
+        put_tiled(weights[t++], (int)F, (int)d, (int)F, p);
+        p += b_gu;
+        w.wd = (const bf16*)p;
+        put_tiled(weights[t++], (int)d, (int)F, 0, p);
+        p += b_d;
     }
     m->final_norm = (const float*)put(weights[t++], d, false, b_norm);
-    m->lm_head = (const bf16*)put(weights[t++], V * d, true, b_embed);
+    m->lm_head = (const bf16*)p;
+    put_tiled(weights[t++], (int)V, (int)d, 0, p);
+    p += b_lm;
     if (rc == ANPD_OK && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
+    if (stage) cudaFree(stage);
     m->d_plan_tables = nullptr;
     if (rc == ANPD_OK) rc = model_make_plans(m);
     if (rc != ANPD_OK) { cudaFree(m->d_plan_tables); cudaFree(m->slab); delete m; return rc; }
@@ -267,10 +298,13 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     kv->max_len = kv->pages_per_seq * KV_PAGE;
     kv->total_pages = kv->pages_per_seq * batch;
     kv->staged = false;
+    kv->warm = false;
+    // the legacy default stream cannot be captured: steps on it are launched one kernel at a time
+    kv->use_graphs = std::getenv("ANPD_NO_GRAPH") == nullptr && m->stream != nullptr && m->stream != cudaStreamLegacy;
     kv->h_kv_len.assign(batch, 0);
     Workspace& ws = kv->ws;
     ws.r_max = std::max(PREFILL_ROWS, batch * ANPD_ROWS);
-    ws.n_max_out = std::max(std::max(m->nqkv, 2 * c.d_ffn), std::max(c.d_model, c.vocab));
+    ws.n_max_out = (std::max(std::max(m->nqkv, 2 * c.d_ffn), std::max(c.d_model, c.vocab)) + 127) / 128 * 128;
     ws.splits_max = m->max_segs;
     ws.amax_blocks = (c.vocab + 1023) / 1024;
     const size_t R = ws.r_max, d = c.d_model, F = c.d_ffn, V = c.vocab, hd = c.head_dim, half = hd / 2;
@@ -362,6 +396,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
 anpd_status anpd_kv_destroy(anpd_kv* kv) {
     if (!kv) return ANPD_ERR_ARG;
     cudaStreamSynchronize(kv->m->stream);
+    for (auto& g : kv->graphs) cudaGraphExecDestroy(g.second.exec);
     cudaFreeHost(kv->h_seq);
     cudaFree(kv->slab);
     delete kv;
@@ -473,15 +508,57 @@ anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_to
     return ANPD_OK;
 }
 
-static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs) {
+// One draft-and-verify step for every sequence of the kv handle, enqueued on the model's stream.
+// K > 0: fold the last step's tokens into the n-gram tables and draft K tokens; K == 0: plain greedy
+// (the confirmed token alone); K < 0: the step's inputs were staged by the host.  Then the forward over
+// the batch * 8 rows, argmax / accept and, in COMMIT mode, the KV commit and token-buffer append.
+// Steps of one shape are captured once into a CUDA graph and replayed.
+static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K = -1) {
     int max_pos = 0;
     for (int b = 0; b < kv->batch; ++b) {
         if (kv->h_kv_len[b] + ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
         max_pos = std::max(max_pos, kv->h_kv_len[b] + ANPD_ROWS - 1);
     }
-    ANPD_TRY(plan_decode_enqueue(m, kv));
-    ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
-    ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
+    cudaStream_t st = m->stream;
+    auto enqueue = [&]() -> anpd_status {
+        if (K > 0) ANPD_TRY(ngram_enqueue_step(d_ctxs, kv->seq, kv->batch, K, st, &m->prof));
+        else if (K == 0) { LAUNCH(&m->prof, st, KC_OTHER, 0, (greedy_stage_kernel<<<kv->batch, 1, 0, st>>>(kv->seq))); }
+        ANPD_TRY(plan_decode_enqueue(m, kv));
+        ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
+        ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
+        return ANPD_OK;
+    };
+    if (m->prof.on || !kv->use_graphs || !kv->warm) {
+        kv->warm = true;
+        return enqueue();
+    }
+    const uint64_t key = (uint64_t)(max_pos / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)mode << 24) |
+                         ((uint64_t)(want_logits ? 1 : 0) << 28) | ((uint64_t)(d_ctxs ? 1 : 0) << 29);
+    auto it = kv->graphs.find(key);
+    if (it == kv->graphs.end()) {
+        const long long before = g_launch_count;
+        cudaGraph_t graph = nullptr;
+        if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+            cudaGetLastError();
+            kv->use_graphs = false;
+            return enqueue();
+        }
+        const anpd_status rc = enqueue();
+        const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+        const int launches = (int)(g_launch_count - before);
+        g_launch_count = before;                      // capturing runs nothing
+        anpd_kv::StepGraph sg{nullptr, launches};
+        if (rc != ANPD_OK || ce != cudaSuccess || !graph || cudaGraphInstantiate(&sg.exec, graph, 0) != cudaSuccess) {
+            cudaGetLastError();
+            if (graph) cudaGraphDestroy(graph);
+            kv->use_graphs = false;                   // fall back to plain launches for good
+            return enqueue();
+        }
+        cudaGraphDestroy(graph);
+        it = kv->graphs.emplace(key, sg).first;
+    }
+    CUDA_TRY(cudaGraphLaunch(it->second.exec, st));
+    g_launch_count += it->second.launches;
     return ANPD_OK;
 }
 
@@ -582,9 +659,7 @@ static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* 
         for (int b = 0; b < B; ++b) ANPD_TRY(seq_error_status(kv->h_seq[b]));
         bool any_active = true;
         while (any_active) {
-            if (K > 0) ANPD_TRY(ngram_enqueue_step(kv->d_ctxs, kv->seq, B, K, st, &m->prof));
-            else { LAUNCH(&m->prof, st, KC_OTHER, 0, (greedy_stage_kernel<<<B, 1, 0, st>>>(kv->seq))); }
-            ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs));
+            ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs, K));
             ANPD_TRY(read_seqs(kv));
             any_active = false;
             for (int b = 0; b < B; ++b) {
@@ -668,10 +743,11 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
         float h; std::memcpy(&h, &u, 4);
         lo[i] = f32_to_bf16_host(a[i] - h);
     }
-    const size_t wb = up256((size_t)N * K * 2), ab = up256((size_t)rows * K * 2), pb = up256((size_t)segs * rows * N * 4),
-                 tb = up256((size_t)plan.m_tiles * 4);
+    const size_t wb = up256(gemm_tiled_elems(N, K) * 2), ab = up256((size_t)rows * K * 2), pb = up256((size_t)segs * rows * N * 4),
+                 tb = up256((size_t)plan.m_tiles * 4), sb = up256((size_t)N * K * 2);
     char* slab = nullptr;
-    if (cudaMalloc((void**)&slab, wb + 2 * ab + pb + tb + 256) != cudaSuccess) { cudaGetLastError(); return ANPD_ERR_OOM; }
+    if (cudaMalloc((void**)&slab, wb + 2 * ab + pb + tb + 256 + sb) != cudaSuccess) { cudaGetLastError(); return ANPD_ERR_OOM; }
+    void* dsrc = slab + wb + 2 * ab + pb + tb + 256;
     bf16* dW = (bf16*)slab; bf16* dhi = (bf16*)(slab + wb); bf16* dlo = (bf16*)(slab + wb + ab);
     float* dpart = (float*)(slab + wb + 2 * ab);
     int* dfirst = (int*)(slab + wb + 2 * ab + pb);
@@ -679,8 +755,10 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
     plan.d_first_cta = dfirst;
     anpd_status rc = ANPD_OK;
     auto body = [&]() -> anpd_status {
+        CUDA_TRY(cudaMemset(slab, 0, wb));
         CUDA_TRY(cudaMemset(slab + wb + 2 * ab, 0, pb + tb + 256));
-        CUDA_TRY(cudaMemcpy(dW, w_bf16, (size_t)N * K * 2, cudaMemcpyHostToDevice));
+        CUDA_TRY(cudaMemcpy(dsrc, w_bf16, (size_t)N * K * 2, cudaMemcpyHostToDevice));
+        ANPD_TRY(gemm_retile_enqueue(dsrc, false, N, K, 0, dW, 0));
         CUDA_TRY(cudaMemcpy(dhi, hi.data(), hi.size() * 2, cudaMemcpyHostToDevice));
         CUDA_TRY(cudaMemcpy(dlo, lo.data(), lo.size() * 2, cudaMemcpyHostToDevice));
         CUDA_TRY(cudaMemcpy(dfirst, plan.first_cta.data(), (size_t)plan.m_tiles * 4, cudaMemcpyHostToDevice));
@@ -688,7 +766,7 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
             ANPD_TRY(gemm_plain_enqueue(dW, dhi, dlo, rows, N, K, dpart, N, 0, nullptr));
         } else {
             CUtensorMap mw, mh, ml;
-            ANPD_TRY(make_tmap_bf16(&mw, dW, N, K, 128, true));
+            ANPD_TRY(make_tmap_tiled(&mw, dW, N, K));
             ANPD_TRY(make_tmap_bf16(&mh, dhi, rows, K, NB, false));
             ANPD_TRY(make_tmap_bf16(&ml, dlo, rows, K, NB, false));
             ANPD_TRY(gemm_tc_enqueue(plan, mw, mh, ml, rows, NB, dpart, (size_t)rows * N, N, derr, 0, nullptr));

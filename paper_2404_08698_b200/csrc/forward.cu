@@ -69,50 +69,102 @@ __global__ void plan_prefill_kernel(const int* prompt, int seq, int start, int p
 
 // ---------------------------------------------------------------------------------------------
 // embedding gather + first RMSNorm;  residual add + RMSNorm
+// One 1024-thread block per row; every thread owns float4 chunks of the row and issues all of a
+// chunk's loads (residual + every partial sum) before using any of them, so the kernel costs about
+// one memory round trip.  The sum of squares is reduced in a fixed tree.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) embed_norm_kernel(const bf16* __restrict__ embed, const int* __restrict__ row_tok,
-                                                         const float* __restrict__ gain, float eps, int d,
-                                                         float* __restrict__ x, bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
-    __shared__ float red[8];
-    const int row = blockIdx.x;
+constexpr int NORM_THREADS = 1024;
+constexpr int NORM_MAX_CHUNKS = 4;        // float4 chunks per thread: rows up to 16384 wide
+
+__device__ __forceinline__ float block_sum_1024(float v, float* red /*[32]*/) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = red[threadIdx.x & 31];
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    __syncthreads();
+    return t;
+}
+
+__device__ __forceinline__ void store_split4(const float4 v, bf16* hi_ptr, bf16* lo_ptr) {
+    bf16 h[4], l[4];
+    split_bf16(v.x, h[0], l[0]); split_bf16(v.y, h[1], l[1]); split_bf16(v.z, h[2], l[2]); split_bf16(v.w, h[3], l[3]);
+    *(uint2*)hi_ptr = *(const uint2*)h;
+    *(uint2*)lo_ptr = *(const uint2*)l;
+}
+
+__global__ void __launch_bounds__(NORM_THREADS) embed_norm_kernel(const bf16* __restrict__ embed, const int* __restrict__ row_tok,
+                                                                  const float* __restrict__ gain, float eps, int d,
+                                                                  float* __restrict__ x, bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
+    __shared__ float red[32];
+    const int row = blockIdx.x, chunks = d >> 2;
     const bf16* e = embed + (size_t)row_tok[row] * d;
-    float* xr = x + (size_t)row * d;
+    float4 v[NORM_MAX_CHUNKS];
     float ss = 0.0f;
-    for (int i = threadIdx.x; i < d; i += 256) {
-        const float v = __bfloat162float(e[i]);
-        xr[i] = v;
-        ss += v * v;
+#pragma unroll
+    for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
+        const int c = threadIdx.x + u * NORM_THREADS;
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < chunks) {
+            const uint2 raw = *(const uint2*)(e + 4 * c);
+            const bf16* b = (const bf16*)&raw;
+            v[u] = make_float4(__bfloat162float(b[0]), __bfloat162float(b[1]), __bfloat162float(b[2]), __bfloat162float(b[3]));
+            *(float4*)(x + (size_t)row * d + 4 * c) = v[u];
+            ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
+        }
     }
-    const float rstd = rsqrtf(block_sum_256(ss, red) / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += 256) {
-        bf16 hi, lo;
-        split_bf16(xr[i] * rstd * gain[i], hi, lo);
-        h_hi[(size_t)row * d + i] = hi;
-        h_lo[(size_t)row * d + i] = lo;
+    const float rstd = rsqrtf(block_sum_1024(ss, red) / (float)d + eps);
+#pragma unroll
+    for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
+        const int c = threadIdx.x + u * NORM_THREADS;
+        if (c < chunks) {
+            const float4 g = *(const float4*)(gain + 4 * c);
+            store_split4(make_float4(v[u].x * rstd * g.x, v[u].y * rstd * g.y, v[u].z * rstd * g.z, v[u].w * rstd * g.w),
+                         h_hi + (size_t)row * d + 4 * c, h_lo + (size_t)row * d + 4 * c);
+        }
     }
 }
 
-// x[row] += sum over splits of part[s][row]; then h = rmsnorm(x) * gain, split into hi + lo.
-__global__ void __launch_bounds__(256) resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part, const int* __restrict__ seg_count,
-                                                         size_t split_stride, int ld_part, const float* __restrict__ gain,
-                                                         float eps, int d, bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
-    __shared__ float red[8];
-    const int row = blockIdx.x;
-    float* xr = x + (size_t)row * d;
+// x[row] += sum of the tile's partial sums (in segment order); then h = rmsnorm(x) * gain as hi + lo.
+__global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part,
+                                                                  const int* __restrict__ seg_count, size_t split_stride, int ld_part,
+                                                                  const float* __restrict__ gain, float eps, int d,
+                                                                  bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
+    __shared__ float red[32];
+    const int row = blockIdx.x, chunks = d >> 2;
+    float4 v[NORM_MAX_CHUNKS];
     float ss = 0.0f;
-    for (int i = threadIdx.x; i < d; i += 256) {
-        float v = xr[i];
-        const int ns = seg_count[i >> 7];
-        for (int s = 0; s < ns; ++s) v += part[s * split_stride + (size_t)row * ld_part + i];
-        xr[i] = v;
-        ss += v * v;
+#pragma unroll
+    for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
+        const int c = threadIdx.x + u * NORM_THREADS;
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < chunks) {
+            const int ns = seg_count[(4 * c) >> 7];
+            const float* pr = part + (size_t)row * ld_part + 4 * c;
+            float4 acc = *(const float4*)(x + (size_t)row * d + 4 * c);
+            for (int s0 = 0; s0 < ns; s0 += 8) {
+                float4 p[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    p[k] = (s0 + k < ns) ? *(const float4*)(pr + (size_t)(s0 + k) * split_stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (s0 + k < ns) { acc.x += p[k].x; acc.y += p[k].y; acc.z += p[k].z; acc.w += p[k].w; }
+            }
+            v[u] = acc;
+            *(float4*)(x + (size_t)row * d + 4 * c) = acc;
+            ss += acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
+        }
     }
-    const float rstd = rsqrtf(block_sum_256(ss, red) / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += 256) {
-        bf16 hi, lo;
-        split_bf16(xr[i] * rstd * gain[i], hi, lo);
-        h_hi[(size_t)row * d + i] = hi;
-        h_lo[(size_t)row * d + i] = lo;
+    const float rstd = rsqrtf(block_sum_1024(ss, red) / (float)d + eps);
+#pragma unroll
+    for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
+        const int c = threadIdx.x + u * NORM_THREADS;
+        if (c < chunks) {
+            const float4 g = *(const float4*)(gain + 4 * c);
+            store_split4(make_float4(v[u].x * rstd * g.x, v[u].y * rstd * g.y, v[u].z * rstd * g.z, v[u].w * rstd * g.w),
+                         h_hi + (size_t)row * d + 4 * c, h_lo + (size_t)row * d + 4 * c);
+        }
     }
 }
 
@@ -145,129 +197,207 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
     const bool is_k = head < Hq + Hkv;
     const int kvh = is_k ? head - Hq : head - Hq - Hkv;
     const int page = page_table[row_seq[row] * pages_per_seq + pos / KV_PAGE];
-    bf16* dst = (is_k ? kpool_l : vpool_l) + (((size_t)page * Hkv + kvh) * KV_PAGE + (pos % KV_PAGE)) * hd;
-    dst[i] = __float2bfloat16_rn(a);
-    dst[i + half] = __float2bfloat16_rn(b);
+    bf16* pg = (is_k ? kpool_l : vpool_l) + ((size_t)page * Hkv + kvh) * KV_PAGE * hd;
+    if (is_k) {                                   // K page: [position][dim]
+        pg[(size_t)(pos % KV_PAGE) * hd + i] = __float2bfloat16_rn(a);
+        pg[(size_t)(pos % KV_PAGE) * hd + i + half] = __float2bfloat16_rn(b);
+    } else {                                      // V page is kept transposed: [dim][position]
+        pg[(size_t)i * KV_PAGE + (pos % KV_PAGE)] = __float2bfloat16_rn(a);
+        pg[(size_t)(i + half) * KV_PAGE + (pos % KV_PAGE)] = __float2bfloat16_rn(b);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
 // attention: per (key page, kv head, group of 8 rows) partial softmax, then a combine in page order
+//
+// The partial kernel works on tensor cores (mma.sync m16n8k16, bf16 in, fp32 out) straight from
+// global memory: a K page is [128 keys][hd] and a V page is stored transposed, [hd][128 keys], so both
+// are the "column" operand of an MMA and each thread fetches 16 contiguous bytes per fragment.  The
+// 8 rows x G query heads that share a kv head are the MMA's 16-row tiles.  q and the softmax weights
+// enter as two bf16 terms each (hi + lo), so only the cache's own bf16 rounding is left.  A warp walks
+// its 32-key blocks in position order with a running (max, sum, output); warps that split a page are
+// merged in block order; pages are merged by the combine kernel in page order.  Every one of these
+// orders is a function of absolute key positions only, and a masked key contributes an exact zero,
+// so a row's result does not depend on which other rows share the launch.
+//
+// Fragment bookkeeping (g = lane / 4, t = lane % 4): a 16-byte load gives a thread 8 consecutive
+// elements e0..e7 of the contraction dimension; (e0,e1),(e2,e3) feed one MMA and (e4,e5),(e6,e7) a
+// second one, and the other operand is permuted the same way, which leaves the sum unchanged.  For
+// QK^T the key a thread column maps to is chosen so that the score fragments are, as they stand,
+// the P fragments the PV product needs: logical key 8j + 2t + e of a block is actual key 8t + 2j + e.
 // ---------------------------------------------------------------------------------------------
-template <int HD>
-__global__ void __launch_bounds__(256) attn_partial_kernel(const float* __restrict__ q, const bf16* __restrict__ kpool_l,
-                                                           const bf16* __restrict__ vpool_l, const int* __restrict__ page_table,
-                                                           int pages_per_seq, const int* __restrict__ row_pos,
-                                                           const int* __restrict__ row_seq, int Hq, int Hkv, float scale,
-                                                           float* __restrict__ pm, float* __restrict__ pl, float* __restrict__ po) {
-    constexpr int KP = HD + 8;                 // padded K row (elements): 16-byte reads stay conflict-free
-    extern __shared__ __align__(16) unsigned char smem[];
-    const int G = Hq / Hkv, NQ = ANPD_ROWS * G;
-    bf16* Ks = (bf16*)smem;                                   // [KV_PAGE][KP]
-    bf16* Vs = Ks + KV_PAGE * KP;                             // [KV_PAGE][HD]
-    float* qs = (float*)(Vs + KV_PAGE * HD);                  // [NQ][HD]
-    float* S = qs + NQ * HD;                                  // [NQ][KV_PAGE]
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
-    const int c = blockIdx.x, g = blockIdx.y, r0 = blockIdx.z * ANPD_ROWS;
+// (x, y) -> packed bf16 pair of the high parts; `lo` receives the packed pair of the remainders.
+__device__ __forceinline__ uint32_t pack_split(float x, float y, uint32_t& lo) {
+    const bf16 hx = __float2bfloat16_rn(x), hy = __float2bfloat16_rn(y);
+    const bf16 lx = __float2bfloat16_rn(x - __bfloat162float(hx)), ly = __float2bfloat16_rn(y - __bfloat162float(hy));
+    lo = (uint32_t)__bfloat16_as_ushort(lx) | ((uint32_t)__bfloat16_as_ushort(ly) << 16);
+    return (uint32_t)__bfloat16_as_ushort(hx) | ((uint32_t)__bfloat16_as_ushort(hy) << 16);
+}
+
+constexpr int ATTN_THREADS = 128;
+constexpr int KEY_BLOCK = 32;
+
+template <int HD>
+__global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float* __restrict__ q, const bf16* __restrict__ kpool_l,
+                                                                    const bf16* __restrict__ vtpool_l, const int* __restrict__ page_table,
+                                                                    int pages_per_seq, const int* __restrict__ row_pos,
+                                                                    const int* __restrict__ row_seq, int Hq, int Hkv, float scale,
+                                                                    float* __restrict__ pm, float* __restrict__ pl, float* __restrict__ po) {
+    constexpr int SLABS = HD / 32;            // 32-wide slabs of the head dimension (two MMAs each)
+    constexpr int DT = HD / 8;                // 8-wide tiles of the head dimension for P V
+    constexpr int OP = HD + 4;                // padded row of the merge buffer
+    __shared__ float sm_m[4][16], sm_l[4][16];
+    __shared__ float sm_o[4][16][OP];
+
+    const int G = Hq / Hkv;
+    const int MT = (ANPD_ROWS * G + 15) / 16;             // 16-row tiles of query vectors: 1, 1, 2, 4 for G = 1, 2, 4, 8
+    const int KG = 4 / MT;                                // warps that split the page's four key blocks
+    const int c = blockIdx.x, kvh = blockIdx.y, r0 = blockIdx.z * ANPD_ROWS;
     const int pos_lo = row_pos[r0], pos_hi = row_pos[r0 + ANPD_ROWS - 1];
     if (c * KV_PAGE > pos_hi) return;
-    const int n_keys = min(KV_PAGE, pos_hi - c * KV_PAGE + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
+    const int mt = warp % MT, kg = warp / MT;
     const int page = page_table[row_seq[r0] * pages_per_seq + c];
-    const bf16* Kg = kpool_l + ((size_t)page * Hkv + g) * KV_PAGE * HD;
-    const bf16* Vg = vpool_l + ((size_t)page * Hkv + g) * KV_PAGE * HD;
-    const int tid = threadIdx.x;
+    const bf16* Kg = kpool_l + ((size_t)page * Hkv + kvh) * KV_PAGE * HD;
+    const bf16* Vg = vtpool_l + ((size_t)page * Hkv + kvh) * KV_PAGE * HD;
 
-    constexpr int VPR = HD / 8;                // 16-byte vectors per row
-    for (int v = tid; v < n_keys * VPR; v += 256) {
-        const int j = v / VPR, w = v % VPR;
-        *(uint4*)(Ks + j * KP + w * 8) = *(const uint4*)(Kg + (size_t)j * HD + w * 8);
-        *(uint4*)(Vs + j * HD + w * 8) = *(const uint4*)(Vg + (size_t)j * HD + w * 8);
+    // this thread's two query vectors (rows gid and gid + 8 of tile mt) and their positions
+    int qpos[2];
+    uint32_t qh[SLABS][2][4], ql[SLABS][2][4];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int qi = mt * 16 + gid + 8 * h;
+        const bool valid = qi < ANPD_ROWS * G;
+        const int r = valid ? qi / G : 0, hl = valid ? qi % G : 0;
+        qpos[h] = valid ? pos_lo + r : -1;                // -1: padding row, sees no key
+        const float* qp = q + (size_t)(r0 + r) * Hq * HD + (size_t)(kvh * G + hl) * HD + 8 * t;
+#pragma unroll
+        for (int s = 0; s < SLABS; ++s) {
+            float4 f0 = make_float4(0.f, 0.f, 0.f, 0.f), f1 = f0;
+            if (valid) { f0 = *(const float4*)(qp + 32 * s); f1 = *(const float4*)(qp + 32 * s + 4); }
+            // first MMA of the slab: elements 0..3; second: elements 4..7.  Register h holds row gid + 8h
+            // for logical k = 2t, 2t+1; register 2 + h the same row for logical k = 2t+8, 2t+9.
+            qh[s][0][h] = pack_split(f0.x * scale, f0.y * scale, ql[s][0][h]);
+            qh[s][0][2 + h] = pack_split(f0.z * scale, f0.w * scale, ql[s][0][2 + h]);
+            qh[s][1][h] = pack_split(f1.x * scale, f1.y * scale, ql[s][1][h]);
+            qh[s][1][2 + h] = pack_split(f1.z * scale, f1.w * scale, ql[s][1][2 + h]);
+        }
     }
-    for (int v = tid; v < NQ * HD; v += 256) {
-        const int qi = v / HD, dim = v % HD;
-        const int r = qi / G, hl = qi % G;
-        qs[v] = q[(size_t)(r0 + r) * Hq * HD + (g * G + hl) * HD + dim] * scale;
-    }
-    __syncthreads();
 
-    // scores: thread = (key j, half of the query vectors), four query vectors at a time
-    {
-        const int j = tid & (KV_PAGE - 1), part = tid >> 7;
-        const int q_lo = part * (NQ / 2), q_hi = q_lo + NQ / 2;
-        const int key_pos = c * KV_PAGE + j;
-        for (int qb = q_lo; qb < q_hi; qb += 4) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            if (j < n_keys) {
-                for (int w = 0; w < VPR; ++w) {
-                    const uint4 kv = *(const uint4*)(Ks + j * KP + w * 8);
-                    const bf16* k8 = (const bf16*)&kv;
-                    float kf[8];
+    float m_run[2] = {-CUDART_INF_F, -CUDART_INF_F}, l_run[2] = {0.f, 0.f};
+    float o[DT][4];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) kf[e] = __bfloat162float(k8[e]);
+    for (int d = 0; d < DT; ++d) { o[d][0] = 0.f; o[d][1] = 0.f; o[d][2] = 0.f; o[d][3] = 0.f; }
+
+    for (int blk = kg; blk < KV_PAGE / KEY_BLOCK; blk += KG) {
+        const int kb0 = c * KV_PAGE + blk * KEY_BLOCK;
+        if (kb0 > pos_hi) break;
+        // ---- scores of 16 query vectors x 32 keys ----
+        float sc[4][4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float4 qa = *(const float4*)(qs + (qb + u) * HD + w * 8);
-                        const float4 qc = *(const float4*)(qs + (qb + u) * HD + w * 8 + 4);
-                        float a = acc[u];
-                        a = fmaf(qa.x, kf[0], a); a = fmaf(qa.y, kf[1], a); a = fmaf(qa.z, kf[2], a); a = fmaf(qa.w, kf[3], a);
-                        a = fmaf(qc.x, kf[4], a); a = fmaf(qc.y, kf[5], a); a = fmaf(qc.z, kf[6], a); a = fmaf(qc.w, kf[7], a);
-                        acc[u] = a;
-                    }
+        for (int j = 0; j < 4; ++j) {
+            sc[j][0] = 0.f; sc[j][1] = 0.f; sc[j][2] = 0.f; sc[j][3] = 0.f;
+            const int key_local = blk * KEY_BLOCK + 8 * (gid >> 1) + 2 * j + (gid & 1);
+            const bf16* kr = Kg + (size_t)key_local * HD + 8 * t;
+#pragma unroll
+            for (int s = 0; s < SLABS; ++s) {
+                const uint4 kv = *(const uint4*)(kr + 32 * s);
+                mma_bf16_16816(sc[j], qh[s][0], kv.x, kv.y);
+                mma_bf16_16816(sc[j], ql[s][0], kv.x, kv.y);
+                mma_bf16_16816(sc[j], qh[s][1], kv.z, kv.w);
+                mma_bf16_16816(sc[j], ql[s][1], kv.z, kv.w);
+            }
+        }
+        // ---- running softmax per row; sc[j][2h + e] belongs to row h, actual key kb0 + 8t + 2j + e ----
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float mx = -CUDART_INF_F;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = kb0 + 8 * t + 2 * j + e;
+                    const float v = (key <= qpos[h]) ? sc[j][2 * h + e] : -CUDART_INF_F;
+                    sc[j][2 * h + e] = v;
+                    mx = fmaxf(mx, v);
                 }
-            }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[h], mx);
+            const bool none = (m_new == -CUDART_INF_F);
+            const float resc = none ? 1.0f : expf(m_run[h] - m_new);
+            float psum = 0.0f;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int r = (qb + u) / G;
-                const bool visible = (j < n_keys) && (key_pos <= pos_lo + r);
-                S[(qb + u) * KV_PAGE + j] = visible ? acc[u] : -CUDART_INF_F;
-            }
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const float p = none ? 0.0f : expf(sc[j][2 * h + e] - m_new);
+                    sc[j][2 * h + e] = p;
+                    psum += p;
+                }
+            psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+            psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+            l_run[h] = l_run[h] * resc + psum;
+            m_run[h] = m_new;
+#pragma unroll
+            for (int d = 0; d < DT; ++d) { o[d][2 * h] *= resc; o[d][2 * h + 1] *= resc; }
+        }
+        // ---- P fragments (hi + lo) for the two MMAs over this block's 32 keys ----
+        uint32_t ph[2][4], plo[2][4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            ph[u][0] = pack_split(sc[2 * u][0], sc[2 * u][1], plo[u][0]);            // row gid,     keys 8t + 4u + {0,1}
+            ph[u][1] = pack_split(sc[2 * u][2], sc[2 * u][3], plo[u][1]);            // row gid + 8
+            ph[u][2] = pack_split(sc[2 * u + 1][0], sc[2 * u + 1][1], plo[u][2]);    // row gid,     keys 8t + 4u + {2,3}
+            ph[u][3] = pack_split(sc[2 * u + 1][2], sc[2 * u + 1][3], plo[u][3]);    // row gid + 8
+        }
+        // ---- O += P V : V^T rows are head dimensions, 16 bytes = keys 8t .. 8t+7 of the block ----
+#pragma unroll
+        for (int d = 0; d < DT; ++d) {
+            const uint4 vv = *(const uint4*)(Vg + (size_t)(8 * d + gid) * KV_PAGE + blk * KEY_BLOCK + 8 * t);
+            mma_bf16_16816(o[d], ph[0], vv.x, vv.y);
+            mma_bf16_16816(o[d], plo[0], vv.x, vv.y);
+            mma_bf16_16816(o[d], ph[1], vv.z, vv.w);
+            mma_bf16_16816(o[d], plo[1], vv.z, vv.w);
         }
     }
-    __syncthreads();
 
-    // softmax pieces per query vector: one warp each, fixed reduction tree
-    {
-        const int warp = tid >> 5, lane = tid & 31;
-        for (int qi = warp; qi < NQ; qi += 8) {
-            float* s = S + qi * KV_PAGE;
-            float m = -CUDART_INF_F;
-            for (int j = lane; j < KV_PAGE; j += 32) m = fmaxf(m, s[j]);
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            float l = 0.0f;
-            for (int j = lane; j < KV_PAGE; j += 32) {
-                const float p = (m == -CUDART_INF_F) ? 0.0f : expf(s[j] - m);
-                s[j] = p;
-                l += p;
-            }
-            for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-            if (lane == 0) {
-                const int r = qi / G, hl = qi % G;
-                const size_t idx = ((size_t)(r0 + r) * Hq + (g * G + hl)) * pages_per_seq + c;
-                pm[idx] = m;
-                pl[idx] = l;
-            }
-        }
+    // ---- merge the warps that split this page (block order), write the page's partial ----
+    if (t == 0) {
+        sm_m[warp][gid] = m_run[0]; sm_m[warp][gid + 8] = m_run[1];
+        sm_l[warp][gid] = l_run[0]; sm_l[warp][gid + 8] = l_run[1];
+    }
+#pragma unroll
+    for (int d = 0; d < DT; ++d) {
+        sm_o[warp][gid][8 * d + 2 * t] = o[d][0];
+        sm_o[warp][gid][8 * d + 2 * t + 1] = o[d][1];
+        sm_o[warp][gid + 8][8 * d + 2 * t] = o[d][2];
+        sm_o[warp][gid + 8][8 * d + 2 * t + 1] = o[d][3];
     }
     __syncthreads();
-
-    // weighted values: thread = (pair of dims, subset of query vectors), keys in position order
-    {
-        constexpr int TPQ = HD / 2;            // threads covering one query vector
-        constexpr int QSUB = 256 / TPQ;        // query-vector subsets
-        const int dp = tid % TPQ, sub = tid / TPQ;
-        for (int qi = sub; qi < NQ; qi += QSUB) {
-            float o0 = 0.0f, o1 = 0.0f;
-            const float* s = S + qi * KV_PAGE;
-            for (int j = 0; j < n_keys; ++j) {
-                const __nv_bfloat162 v2 = *(const __nv_bfloat162*)(Vs + j * HD + 2 * dp);
-                const float p = s[j];
-                o0 = fmaf(p, __low2float(v2), o0);
-                o1 = fmaf(p, __high2float(v2), o1);
-            }
-            const int r = qi / G, hl = qi % G;
-            const size_t idx = ((size_t)(r0 + r) * Hq + (g * G + hl)) * pages_per_seq + c;
-            po[idx * HD + 2 * dp] = o0;
-            po[idx * HD + 2 * dp + 1] = o1;
+    for (int idx = threadIdx.x; idx < MT * 16 * HD; idx += ATTN_THREADS) {
+        const int dim = idx % HD, rowi = (idx / HD) % 16, tile = idx / (HD * 16);
+        const int qi = tile * 16 + rowi;
+        if (qi >= ANPD_ROWS * G) continue;
+        float M = -CUDART_INF_F;
+        for (int k = 0; k < KG; ++k) M = fmaxf(M, sm_m[k * MT + tile][rowi]);
+        float L = 0.0f, O = 0.0f;
+        for (int k = 0; k < KG; ++k) {
+            const float mk = sm_m[k * MT + tile][rowi];
+            const float w = (mk == -CUDART_INF_F) ? 0.0f : expf(mk - M);
+            L = fmaf(sm_l[k * MT + tile][rowi], w, L);
+            O = fmaf(sm_o[k * MT + tile][rowi][dim], w, O);
         }
+        const int r = qi / G, hl = qi % G;
+        const size_t out = ((size_t)(r0 + r) * Hq + (kvh * G + hl)) * pages_per_seq + c;
+        po[out * HD + dim] = O;
+        if (dim == 0) { pm[out] = M; pl[out] = L; }
     }
 }
 
@@ -421,11 +551,13 @@ __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict_
                                                          float* __restrict__ part, int ld_part) {
     const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (n >= N) return;
-    const bf16* w = W + (size_t)n * K;
+    // tiled storage: tile (n / 128, k / 64) is 128 x 64 contiguous
+    const int k_blocks = (K + 63) / 64;
+    const bf16* w = W + ((size_t)(n >> 7) * k_blocks * 128 + (n & 127)) * 64;
     for (int r0 = 0; r0 < rows; r0 += 8) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int k0 = lane * 8; k0 < K; k0 += 256) {
-            const uint4 wv = *(const uint4*)(w + k0);
+            const uint4 wv = *(const uint4*)(w + (size_t)(k0 >> 6) * (128 * 64) + (k0 & 63));
             const bf16* w8 = (const bf16*)&wv;
             float wf[8];
 #pragma unroll
@@ -480,21 +612,14 @@ template <int HD>
 anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos) {
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
-    const int G = c.n_q_heads / c.n_kv_heads, NQ = ANPD_ROWS * G;
-    const size_t smem = (size_t)KV_PAGE * (HD + 8) * 2 + (size_t)KV_PAGE * HD * 2 + (size_t)NQ * HD * 4 + (size_t)NQ * KV_PAGE * 4;
-    static bool attr_set = false;
-    if (!attr_set) {
-        CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-        attr_set = true;
-    }
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * HD;
     const int chunks = max_pos / KV_PAGE + 1;
     dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (attn_partial_kernel<HD><<<grid, 256, smem, m->stream>>>(ws.q, kv->kpool + layer * layer_elems, kv->vpool + layer * layer_elems,
-                                                                   kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq,
-                                                                   c.n_q_heads, c.n_kv_heads, 1.0f / sqrtf((float)HD),
-                                                                   ws.attn_m, ws.attn_l, ws.attn_o)));
+           (attn_partial_kernel<HD><<<grid, ATTN_THREADS, 0, m->stream>>>(ws.q, kv->kpool + layer * layer_elems, kv->vpool + layer * layer_elems,
+                                                                         kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq,
+                                                                         c.n_q_heads, c.n_kv_heads, 1.0f / sqrtf((float)HD),
+                                                                         ws.attn_m, ws.attn_l, ws.attn_o)));
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (attn_combine_kernel<<<dim3(rows, c.n_q_heads), HD, 0, m->stream>>>(ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
@@ -550,7 +675,7 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * hd;
     const int* segs = nullptr;
 
-    LAUNCH(pf, st, KC_OTHER, 0, (embed_norm_kernel<<<rows, 256, 0, st>>>(m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
+    LAUNCH(pf, st, KC_OTHER, 0, (embed_norm_kernel<<<rows, NORM_THREADS, 0, st>>>(m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
                                                                       ws.x, ws.h_hi, ws.h_lo)));
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& w = m->layers[l];
@@ -564,7 +689,7 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
         else ANPD_TRY(attn_enqueue<64>(m, kv, l, rows, max_pos));
         ANPD_TRY(gemm_enqueue(m, kv, GK_O, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (resid_norm_kernel<<<rows, 256, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
+               (resid_norm_kernel<<<rows, NORM_THREADS, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
         ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
@@ -573,7 +698,7 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
         ANPD_TRY(gemm_enqueue(m, kv, GK_DOWN, l, rows, &segs));
         const float* next_gain = (l + 1 < c.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
         LAUNCH(pf, st, KC_OTHER, 0,
-               (resid_norm_kernel<<<rows, 256, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
+               (resid_norm_kernel<<<rows, NORM_THREADS, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
     }
     if (!head) { CUDA_TRY(cudaGetLastError()); return ANPD_OK; }

@@ -176,7 +176,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (!ok) break;
                 unsigned char* sa = smem + (size_t)stage * stage_bytes;
                 mbar_expect_tx(&bar_full[stage], (uint32_t)stage_bytes);
-                tma_load_2d(sa, &map_w, kb * TILE_K, tile * TILE_M, &bar_full[stage], pol_w);
+                tma_load_2d(sa, &map_w, 0, (int)(blk * TILE_M), &bar_full[stage], pol_w);       // tile (tile, kb): 16 KB contiguous
                 tma_load_2d(sa + A_BYTES, &map_hi, kb * TILE_K, 0, &bar_full[stage], pol_a);
                 tma_load_2d(sa + A_BYTES + g.NB * 128, &map_lo, kb * TILE_K, 0, &bar_full[stage], pol_a);
                 ++issued;
@@ -275,6 +275,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     if (threadIdx.x == 0 && abort_flag) atomicExch(g.err, GEMM_ERR_TIMEOUT);
 }
 
+template <typename T>
+__global__ void retile_kernel(const T* __restrict__ src, int rows, int K, int row_off, int k_blocks, bf16* __restrict__ dst) {
+    const int chunks = K / 8;                                  // 8 consecutive inputs never straddle a 64-wide block
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)rows * chunks; i += (size_t)gridDim.x * blockDim.x) {
+        const int r = (int)(i / chunks), k0 = (int)(i % chunks) * 8;
+        const int n = row_off + r;
+        bf16* out = dst + ((((size_t)(n >> 7) * k_blocks + (k0 >> 6)) * TILE_M + (n & 127)) * TILE_K + (k0 & 63));
+        const T* in = src + (size_t)r * K + k0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = (bf16)in[e];
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -308,6 +321,25 @@ anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, 
         if (std::getenv("ANPD_VERBOSE")) std::fprintf(stderr, "[anpd] cuTensorMapEncodeTiled failed: %d (rows %d K %d box %d)\n", (int)r, rows, K, box_rows);
         return ANPD_ERR_CUDA;
     }
+    return ANPD_OK;
+}
+
+size_t gemm_tiled_elems(int N, int K) {
+    return (size_t)((N + TILE_M - 1) / TILE_M) * ((K + TILE_K - 1) / TILE_K) * TILE_M * TILE_K;
+}
+
+anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, int N, int K) {
+    const int rows = (int)(gemm_tiled_elems(N, K) / TILE_K);
+    return make_tmap_bf16(out, base_tiled, rows, TILE_K, TILE_M, true);
+}
+
+anpd_status gemm_retile_enqueue(const void* src, bool src_is_f32, int rows, int K, int row_off, bf16* dst_tiled, cudaStream_t st) {
+    const int k_blocks = (K + TILE_K - 1) / TILE_K;
+    const size_t work = (size_t)rows * (K / 8);
+    const int blocks = (int)std::min<size_t>((work + 255) / 256, 148 * 16);
+    if (src_is_f32) retile_kernel<float><<<blocks, 256, 0, st>>>((const float*)src, rows, K, row_off, k_blocks, dst_tiled);
+    else retile_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)src, rows, K, row_off, k_blocks, dst_tiled);
+    CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
 

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <map>
 #include <vector>
 
 #include "anpd.h"
@@ -141,6 +142,7 @@ struct GemmPlan {
 enum GemmKind { GK_QKV = 0, GK_O = 1, GK_GU = 2, GK_DOWN = 3, GK_LM = 4, GK_COUNT = 5 };
 
 struct LayerW {
+    // all four matrices in tiled storage (see gemm_tiled_elems)
     const __nv_bfloat16* wqkv;        // [(Hq + 2 Hkv) * hd, d]  (q rows, then k rows, then v rows)
     const __nv_bfloat16* wo;          // [d, Hq * hd]
     const __nv_bfloat16* wgu;         // [2 F, d]  (gate rows, then up rows)
@@ -155,7 +157,7 @@ struct anpd_model {
     cudaStream_t stream;
     int dq, dkv, nqkv;
     const __nv_bfloat16* embed;       // [V, d]
-    const __nv_bfloat16* lm_head;     // [V, d]
+    const __nv_bfloat16* lm_head;     // [V, d], tiled storage
     const float* final_norm;          // [d]
     std::vector<LayerW> layers;
     void* slab;
@@ -195,7 +197,7 @@ struct Workspace {
 struct anpd_kv {
     anpd_model* m;
     int batch, max_len, pages_per_seq, total_pages;
-    __nv_bfloat16 *kpool, *vpool;     // [L][total_pages][Hkv][KV_PAGE][hd]
+    __nv_bfloat16 *kpool, *vpool;     // per layer and page: K [Hkv][KV_PAGE][hd]; V transposed [Hkv][hd][KV_PAGE]
     int* page_table;                  // device [batch][pages_per_seq]
     float *rope_cos, *rope_sin;       // [max_len][hd/2]
     SeqState* seq;                    // device [batch]
@@ -208,6 +210,11 @@ struct anpd_kv {
     void* slab;
     size_t slab_bytes;
     bool staged;
+    // one instantiated CUDA graph per distinct step shape (draft length, mode, attention grid)
+    struct StepGraph { cudaGraphExec_t exec; int launches; };
+    std::map<uint64_t, StepGraph> graphs;
+    bool use_graphs;
+    bool warm;                        // the first step runs eagerly (one-time function attributes, lazy module loading)
 };
 
 // Forward over `rows` rows (a multiple of 8; 8 consecutive rows always belong to one sequence and
@@ -226,6 +233,12 @@ anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev*
 
 // gemm_tc.cu
 anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, int box_rows, bool streamed);
+// Weight matrices are stored as a sequence of 128 x 64 tiles, tile (t, kb) at element ((t * k_blocks + kb) * 128) * 64.
+size_t gemm_tiled_elems(int N, int K);
+anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, int N, int K);
+// Scatters rows [row_off, row_off + rows) of a row-major [rows][K] source (bf16, or fp32 rounded to
+// bf16) into the tiled storage of a matrix with K inputs.  The padding must already be zero.
+anpd_status gemm_retile_enqueue(const void* src, bool src_is_f32, int rows, int K, int row_off, __nv_bfloat16* dst_tiled, cudaStream_t st);
 void gemm_make_plan(GemmPlan* p, int N, int K, int num_sms);
 anpd_status gemm_tc_enqueue(const GemmPlan& plan, const CUtensorMap& map_w, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
                             int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,

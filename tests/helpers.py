@@ -15,6 +15,16 @@ def require_gpu():
     build.build()
 
 
+_streams = []
+
+
+def new_stream() -> int:
+    """A non-default CUDA stream handle (steps on such a stream run as replayed CUDA graphs)."""
+    st = torch.cuda.Stream()
+    _streams.append(st)
+    return st.cuda_stream
+
+
 def gpu_model(A, shape, weights, stream: int = 0) -> int:
     return A.anpd_model_create(shape, [weights[n] for n, _ in tensor_shapes(shape)], stream)
 

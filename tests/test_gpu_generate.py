@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import as_bf16_values, check_stream_against_oracle, gpu_model, require_gpu
+from helpers import as_bf16_values, check_stream_against_oracle, gpu_model, new_stream, require_gpu
 from oracle.anpd import anpd_generate as oracle_anpd
 from oracle.decoder import Decoder
 from oracle.mln import MLN
@@ -25,17 +25,18 @@ def A():
 def c1(A):
     wl = WORKLOADS["C1"]
     w = make_weights(wl.shape, wl.weight_seed, wl.weights_bf16)
-    m = gpu_model(A, wl.shape, w)
+    st = new_stream()                                   # a real stream: the loop replays CUDA graphs
+    m = gpu_model(A, wl.shape, w, st)
     kv = A.anpd_kv_create(m, 512)
-    yield wl, w, m, kv
+    yield wl, w, m, kv, st
     A.anpd_kv_destroy(kv)
     A.anpd_model_destroy(m)
 
 
 def test_c1_anpd_equals_greedy_equals_oracle(A, c1):
-    wl, w, m, kv = c1
+    wl, w, m, kv, st = c1
     prompt = make_prompts(wl)[0]
-    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, 512)
+    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, 512, 0, st)
     try:
         out, st = A.anpd_generate(m, kv, ctx, prompt, wl.max_new, wl.K)
         ref, st0 = A.anpd_generate(m, kv, ctx, prompt, wl.max_new, 0)
@@ -59,9 +60,9 @@ def test_c1_anpd_equals_greedy_equals_oracle(A, c1):
 
 
 def test_tables_after_generate_match_oracle_on_the_generated_stream(A, c1):
-    wl, w, m, kv = c1
+    wl, w, m, kv, st = c1
     prompt = make_prompts(wl)[0]
-    ctx = A.anpd_ngram_create(2, 4, 512)
+    ctx = A.anpd_ngram_create(2, 4, 512, 0, st)
     try:
         ref, _ = A.anpd_generate(m, kv, ctx, prompt, 48, 0)             # greedy, a little longer
         out, st = A.anpd_generate(m, kv, ctx, prompt, 40, 5)
@@ -140,12 +141,13 @@ def test_cyclic_copy_model_accepts_every_draft(A):
 def test_batch_equals_independent_runs(A):
     shape = ModelShape(2, 128, 4, 4, 64, 200, 300)
     w = make_weights(shape, 9, False, std=0.08)
-    m = gpu_model(A, shape, w)
+    st = new_stream()
+    m = gpu_model(A, shape, w, st)
     B, plen, M, K = 3, 70, 30, 4
     prompts = np.stack([np.concatenate([markov_prompt(35, shape.vocab, 2, 50 + b)] * 2) for b in range(B)])
     kv1 = A.anpd_kv_create(m, 256, 1)
     kvb = A.anpd_kv_create(m, 256, B, True)
-    ctxs = [A.anpd_ngram_create(2, 4, 256) for _ in range(B)]
+    ctxs = [A.anpd_ngram_create(2, 4, 256, 0, st) for _ in range(B)]
     try:
         singles = [A.anpd_generate(m, kv1, ctxs[0], prompts[b], M, K) for b in range(B)]
         outs, stats = A.anpd_generate_batch(m, kvb, ctxs, prompts, M, K)
@@ -164,8 +166,8 @@ def test_batch_equals_independent_runs(A):
 
 
 def test_generate_error_paths(A, c1):
-    wl, w, m, kv = c1
-    ctx = A.anpd_ngram_create(2, 3, 128)
+    wl, w, m, kv, st = c1
+    ctx = A.anpd_ngram_create(2, 3, 128, 0, st)
     try:
         with pytest.raises(A.AnpdError) as e:
             A.anpd_generate(m, kv, ctx, list(range(100)), 64, 4)         # context too small
