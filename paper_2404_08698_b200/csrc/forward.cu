@@ -210,9 +210,11 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
 // ---------------------------------------------------------------------------------------------
 // attention: per (key page, kv head, group of 8 rows) partial softmax, then a combine in page order
 //
-// The partial kernel works on tensor cores (mma.sync m16n8k16, bf16 in, fp32 out) straight from
-// global memory: a K page is [128 keys][hd] and a V page is stored transposed, [hd][128 keys], so both
-// are the "column" operand of an MMA and each thread fetches 16 contiguous bytes per fragment.  The
+// The partial kernel works on tensor cores (mma.sync m16n8k16, bf16 in, fp32 out).  A K page is
+// [128 keys][hd] and a V page is stored transposed, [hd][128 keys], so both are the "column" operand
+// of an MMA and each thread fetches 16 contiguous bytes per fragment.  A block first issues every
+// 16-byte asynchronous copy of its K and V page into (row-padded, bank-conflict-free) shared memory,
+// so one block keeps up to 64 KB in flight, then computes from shared memory.  The
 // 8 rows x G query heads that share a kv head are the MMA's 16-row tiles.  q and the softmax weights
 // enter as two bf16 terms each (hi + lo), so only the cache's own bf16 rounding is left.  A warp walks
 // its 32-key blocks in position order with a running (max, sum, output); warps that split a page are
@@ -252,8 +254,13 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
     constexpr int SLABS = HD / 32;            // 32-wide slabs of the head dimension (two MMAs each)
     constexpr int DT = HD / 8;                // 8-wide tiles of the head dimension for P V
     constexpr int OP = HD + 4;                // padded row of the merge buffer
+    constexpr int KPITCH = HD * 2 + 64;       // bytes per staged K row (64 bytes of padding: conflict-free 16-byte reads)
+    constexpr int VPITCH = KV_PAGE * 2 + 64;  // bytes per staged V^T row
+    extern __shared__ __align__(16) unsigned char attn_smem[];
+    unsigned char* Ks = attn_smem;                                  // [KV_PAGE][KPITCH]
+    unsigned char* Vs = attn_smem + KV_PAGE * KPITCH;               // [HD][VPITCH]
+    float (*sm_o)[16][OP] = (float (*)[16][OP])Ks;                  // [4][16][OP], reuses the K staging area after the last MMA
     __shared__ float sm_m[4][16], sm_l[4][16];
-    __shared__ float sm_o[4][16][OP];
 
     const int G = Hq / Hkv;
     const int MT = (ANPD_ROWS * G + 15) / 16;             // 16-row tiles of query vectors: 1, 1, 2, 4 for G = 1, 2, 4, 8
@@ -266,6 +273,24 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
     const int page = page_table[row_seq[r0] * pages_per_seq + c];
     const bf16* Kg = kpool_l + ((size_t)page * Hkv + kvh) * KV_PAGE * HD;
     const bf16* Vg = vtpool_l + ((size_t)page * Hkv + kvh) * KV_PAGE * HD;
+
+    // stage the part of the page that any row can see: whole 32-key blocks up to pos_hi
+    {
+        const int nblk = min(KV_PAGE / KEY_BLOCK, (pos_hi - c * KV_PAGE) / KEY_BLOCK + 1);
+        constexpr int KCH = HD * 2 / 16;                  // 16-byte chunks per K row
+        for (int i = threadIdx.x; i < nblk * KEY_BLOCK * KCH; i += ATTN_THREADS) {
+            const int row = i / KCH, ch = i % KCH;
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(Ks + row * KPITCH + ch * 16);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(Kg + (size_t)row * HD + ch * 8) : "memory");
+        }
+        const int vch = nblk * (KEY_BLOCK * 2 / 16);      // chunks per V^T row that hold visible keys
+        for (int i = threadIdx.x; i < HD * vch; i += ATTN_THREADS) {
+            const int row = i / vch, ch = i % vch;
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(Vs + row * VPITCH + ch * 16);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(Vg + (size_t)row * KV_PAGE + ch * 8) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
 
     // this thread's two query vectors (rows gid and gid + 8 of tile mt) and their positions
     int qpos[2];
@@ -294,6 +319,8 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
     float o[DT][4];
 #pragma unroll
     for (int d = 0; d < DT; ++d) { o[d][0] = 0.f; o[d][1] = 0.f; o[d][2] = 0.f; o[d][3] = 0.f; }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
 
     for (int blk = kg; blk < KV_PAGE / KEY_BLOCK; blk += KG) {
         const int kb0 = c * KV_PAGE + blk * KEY_BLOCK;
@@ -304,10 +331,10 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
         for (int j = 0; j < 4; ++j) {
             sc[j][0] = 0.f; sc[j][1] = 0.f; sc[j][2] = 0.f; sc[j][3] = 0.f;
             const int key_local = blk * KEY_BLOCK + 8 * (gid >> 1) + 2 * j + (gid & 1);
-            const bf16* kr = Kg + (size_t)key_local * HD + 8 * t;
+            const unsigned char* kr = Ks + key_local * KPITCH + 16 * t;
 #pragma unroll
             for (int s = 0; s < SLABS; ++s) {
-                const uint4 kv = *(const uint4*)(kr + 32 * s);
+                const uint4 kv = *(const uint4*)(kr + 64 * s);
                 mma_bf16_16816(sc[j], qh[s][0], kv.x, kv.y);
                 mma_bf16_16816(sc[j], ql[s][0], kv.x, kv.y);
                 mma_bf16_16816(sc[j], qh[s][1], kv.z, kv.w);
@@ -360,7 +387,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
         // ---- O += P V : V^T rows are head dimensions, 16 bytes = keys 8t .. 8t+7 of the block ----
 #pragma unroll
         for (int d = 0; d < DT; ++d) {
-            const uint4 vv = *(const uint4*)(Vg + (size_t)(8 * d + gid) * KV_PAGE + blk * KEY_BLOCK + 8 * t);
+            const uint4 vv = *(const uint4*)(Vs + (8 * d + gid) * VPITCH + (blk * KEY_BLOCK + 8 * t) * 2);
             mma_bf16_16816(o[d], ph[0], vv.x, vv.y);
             mma_bf16_16816(o[d], plo[0], vv.x, vv.y);
             mma_bf16_16816(o[d], ph[1], vv.z, vv.w);
@@ -369,6 +396,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
     }
 
     // ---- merge the warps that split this page (block order), write the page's partial ----
+    __syncthreads();                                      // every warp is done reading the staged K rows
     if (t == 0) {
         sm_m[warp][gid] = m_run[0]; sm_m[warp][gid + 8] = m_run[1];
         sm_l[warp][gid] = l_run[0]; sm_l[warp][gid + 8] = l_run[1];
@@ -614,12 +642,19 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     Workspace& ws = kv->ws;
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * HD;
     const int chunks = max_pos / KV_PAGE + 1;
+    const size_t smem = (size_t)KV_PAGE * (HD * 2 + 64) + (size_t)HD * (KV_PAGE * 2 + 64);
+    static_assert(4 * 16 * (HD + 4) * sizeof(float) <= (size_t)KV_PAGE * (HD * 2 + 64), "merge buffer must fit in the K staging area");
+    static bool attr_set = false;
+    if (!attr_set) {
+        CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set = true;
+    }
     dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (attn_partial_kernel<HD><<<grid, ATTN_THREADS, 0, m->stream>>>(ws.q, kv->kpool + layer * layer_elems, kv->vpool + layer * layer_elems,
-                                                                         kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq,
-                                                                         c.n_q_heads, c.n_kv_heads, 1.0f / sqrtf((float)HD),
-                                                                         ws.attn_m, ws.attn_l, ws.attn_o)));
+           (attn_partial_kernel<HD><<<grid, ATTN_THREADS, smem, m->stream>>>(ws.q, kv->kpool + layer * layer_elems, kv->vpool + layer * layer_elems,
+                                                                            kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq,
+                                                                            c.n_q_heads, c.n_kv_heads, 1.0f / sqrtf((float)HD),
+                                                                            ws.attn_m, ws.attn_l, ws.attn_o)));
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (attn_combine_kernel<<<dim3(rows, c.n_q_heads), HD, 0, m->stream>>>(ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));

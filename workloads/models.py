@@ -69,6 +69,8 @@ WORKLOADS = {
     "C3": Workload("C3", S7B, True, 2, 1536, 3, True, 256, 5, 5, 1, 1002),
     # C4 (verify-step microbenchmark) reuses the C3 model; see bench.py
     "C5": Workload("C5", S13B, True, 3, 2048, 3, True, 512, 7, 6, 8, 1004),
+    # two layers of the 7B shape: the per-layer kernels of C3 at a size a profiler capture can hold
+    "C3-2L": Workload("C3-2L", ModelShape(2, 4096, 32, 32, 128, 11008, 32000), True, 2, 1536, 3, True, 256, 5, 5, 1, 1002),
 }
 
 LAYER_TENSORS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
