@@ -109,18 +109,11 @@ bool have_device() {
 // GEMM plans (how each matrix shape is cut across the SMs) and the TMA views of the weights.
 static anpd_status model_make_plans(anpd_model* m) {
     const anpd_model_config& c = m->cfg;
-    int dev = 0, sms = 0;
-    CUDA_TRY(cudaGetDevice(&dev));
-    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    m->num_sms = sms;
     m->plain_gemm = std::getenv("ANPD_PLAIN_GEMM") != nullptr;
-    const int shapes[GK_COUNT][2] = {{m->nqkv, c.d_model}, {c.d_model, m->dq}, {2 * c.d_ffn, c.d_model}, {c.d_model, c.d_ffn},
-                                     {c.vocab, c.d_model}};
     size_t ints = 0;
     int max_tiles = 0;
     m->max_segs = 1;
     for (int k = 0; k < GK_COUNT; ++k) {
-        gemm_make_plan(&m->plan[k], shapes[k][0], shapes[k][1], sms);
         ints += 2 * (size_t)m->plan[k].m_tiles;
         max_tiles = std::max(max_tiles, m->plan[k].m_tiles);
         m->max_segs = std::max(m->max_segs, m->plan[k].max_segs);
@@ -141,12 +134,12 @@ static anpd_status model_make_plans(anpd_model* m) {
     CUDA_TRY(cudaMemcpy(m->d_plan_tables, host.data(), ints * sizeof(int), cudaMemcpyHostToDevice));
     for (int l = 0; l < c.n_layers; ++l) {
         LayerW& w = m->layers[l];
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_QKV], w.wqkv, m->nqkv, c.d_model));
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_O], w.wo, c.d_model, m->dq));
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_GU], w.wgu, 2 * c.d_ffn, c.d_model));
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_DOWN], w.wd, c.d_model, c.d_ffn));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_QKV], w.wqkv, m->plan[GK_QKV]));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_O], w.wo, m->plan[GK_O]));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_GU], w.wgu, m->plan[GK_GU]));
+        ANPD_TRY(make_tmap_tiled(&w.map[GK_DOWN], w.wd, m->plan[GK_DOWN]));
     }
-    ANPD_TRY(make_tmap_tiled(&m->map_lm, m->lm_head, c.vocab, c.d_model));
+    ANPD_TRY(make_tmap_tiled(&m->map_lm, m->lm_head, m->plan[GK_LM]));
     return ANPD_OK;
 }
 
@@ -202,9 +195,19 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     // GEMM weights are stored tile by tile (128 output rows x 64 inputs, 16 KB contiguous each, zero
     // padded at ragged edges) so that every TMA box is one contiguous read; the embedding table stays
     // row-major because it is only gathered.
-    const size_t b_embed = up256(V * d * 2), b_lm = up256(gemm_tiled_elems((int)V, (int)d) * 2),
-                 b_qkv = up256(gemm_tiled_elems(m->nqkv, (int)d) * 2), b_o = up256(gemm_tiled_elems((int)d, m->dq) * 2),
-                 b_gu = up256(gemm_tiled_elems(2 * (int)F, (int)d) * 2), b_d = up256(gemm_tiled_elems((int)d, (int)F) * 2),
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError(); delete m; return ANPD_ERR_CUDA;
+        }
+        m->num_sms = sms;
+        const int shapes[GK_COUNT][2] = {{m->nqkv, c.d_model}, {c.d_model, m->dq}, {2 * c.d_ffn, c.d_model}, {c.d_model, c.d_ffn},
+                                         {c.vocab, c.d_model}};
+        for (int k = 0; k < GK_COUNT; ++k) gemm_make_plan(&m->plan[k], shapes[k][0], shapes[k][1], sms);
+    }
+    const size_t b_embed = up256(V * d * 2), b_lm = up256(gemm_tiled_elems(m->plan[GK_LM]) * 2),
+                 b_qkv = up256(gemm_tiled_elems(m->plan[GK_QKV]) * 2), b_o = up256(gemm_tiled_elems(m->plan[GK_O]) * 2),
+                 b_gu = up256(gemm_tiled_elems(m->plan[GK_GU]) * 2), b_d = up256(gemm_tiled_elems(m->plan[GK_DOWN]) * 2),
                  b_norm = up256(d * 4);
     m->slab_bytes = b_embed + b_lm + b_norm + c.n_layers * (b_qkv + b_o + b_gu + b_d + 2 * b_norm);
     if (cudaMalloc(&m->slab, m->slab_bytes) != cudaSuccess) { cudaGetLastError(); delete m; return ANPD_ERR_OOM; }
@@ -227,7 +230,7 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
         return dst;
     };
     // rows [row_off, row_off + rows) of a tiled [*, K] matrix at dst
-    auto put_tiled = [&](const void* src, int rows, int K, int row_off, void* dst) {
+    auto put_tiled = [&](int kind, const void* src, int rows, int K, int row_off, void* dst) {
         if (rc != ANPD_OK) return;
         const void* dsrc = src;
         if (!dev) {
@@ -235,7 +238,7 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
                 cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; return; }
             dsrc = stage;
         }
-        rc = gemm_retile_enqueue(dsrc, !bf, rows, K, row_off, (bf16*)dst, st);
+        rc = gemm_retile_enqueue(m->plan[kind], dsrc, !bf, rows, row_off, (bf16*)dst, st);
         if (rc == ANPD_OK && !dev && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
     };
     int t = 0;
@@ -246,25 +249,25 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
         w.attn_norm = (const float*)put(weights[t++], d, false, b_norm);
         // q, k and v rows form one matrix so that one GEMM produces all three
         w.wqkv = (const bf16*)p;
-        put_tiled(weights[t++], m->dq, (int)d, 0, p);
-        put_tiled(weights[t++], m->dkv, (int)d, m->dq, p);
-        put_tiled(weights[t++], m->dkv, (int)d, m->dq + m->dkv, p);
+        put_tiled(GK_QKV, weights[t++], m->dq, (int)d, 0, p);
+        put_tiled(GK_QKV, weights[t++], m->dkv, (int)d, m->dq, p);
+        put_tiled(GK_QKV, weights[t++], m->dkv, (int)d, m->dq + m->dkv, p);
         p += b_qkv;
         w.wo = (const bf16*)p;
-        put_tiled(weights[t++], (int)d, m->dq, 0, p);
+        put_tiled(GK_O, weights[t++], (int)d, m->dq, 0, p);
         p += b_o;
         w.ffn_norm = (const float*)put(weights[t++], d, false, b_norm);
         w.wgu = (const bf16*)p;
-        put_tiled(weights[t++], (int)F, (int)d, 0, p);
-        put_tiled(weights[t++], (int)F, (int)d, (int)F, p);
+        put_tiled(GK_GU, weights[t++], (int)F, (int)d, 0, p);
+        put_tiled(GK_GU, weights[t++], (int)F, (int)d, (int)F, p);
         p += b_gu;
         w.wd = (const bf16*)p;
-        put_tiled(weights[t++], (int)d, (int)F, 0, p);
+        put_tiled(GK_DOWN, weights[t++], (int)d, (int)F, 0, p);
         p += b_d;
     }
     m->final_norm = (const float*)put(weights[t++], d, false, b_norm);
     m->lm_head = (const bf16*)p;
-    put_tiled(weights[t++], (int)V, (int)d, 0, p);
+    put_tiled(GK_LM, weights[t++], (int)V, (int)d, 0, p);
     p += b_lm;
     if (rc == ANPD_OK && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
     if (stage) cudaFree(stage);
@@ -743,7 +746,7 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
         float h; std::memcpy(&h, &u, 4);
         lo[i] = f32_to_bf16_host(a[i] - h);
     }
-    const size_t wb = up256(gemm_tiled_elems(N, K) * 2), ab = up256((size_t)rows * K * 2), pb = up256((size_t)segs * rows * N * 4),
+    const size_t wb = up256(gemm_tiled_elems(plan) * 2), ab = up256((size_t)rows * K * 2), pb = up256((size_t)segs * rows * N * 4),
                  tb = up256((size_t)plan.m_tiles * 4), sb = up256((size_t)N * K * 2);
     char* slab = nullptr;
     if (cudaMalloc((void**)&slab, wb + 2 * ab + pb + tb + 256 + sb) != cudaSuccess) { cudaGetLastError(); return ANPD_ERR_OOM; }
@@ -758,15 +761,15 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
         CUDA_TRY(cudaMemset(slab, 0, wb));
         CUDA_TRY(cudaMemset(slab + wb + 2 * ab, 0, pb + tb + 256));
         CUDA_TRY(cudaMemcpy(dsrc, w_bf16, (size_t)N * K * 2, cudaMemcpyHostToDevice));
-        ANPD_TRY(gemm_retile_enqueue(dsrc, false, N, K, 0, dW, 0));
+        ANPD_TRY(gemm_retile_enqueue(plan, dsrc, false, N, 0, dW, 0));
         CUDA_TRY(cudaMemcpy(dhi, hi.data(), hi.size() * 2, cudaMemcpyHostToDevice));
         CUDA_TRY(cudaMemcpy(dlo, lo.data(), lo.size() * 2, cudaMemcpyHostToDevice));
         CUDA_TRY(cudaMemcpy(dfirst, plan.first_cta.data(), (size_t)plan.m_tiles * 4, cudaMemcpyHostToDevice));
         if (plain) {
-            ANPD_TRY(gemm_plain_enqueue(dW, dhi, dlo, rows, N, K, dpart, N, 0, nullptr));
+            ANPD_TRY(gemm_plain_enqueue(plan, dW, dhi, dlo, rows, dpart, N, 0, nullptr));
         } else {
             CUtensorMap mw, mh, ml;
-            ANPD_TRY(make_tmap_tiled(&mw, dW, N, K));
+            ANPD_TRY(make_tmap_tiled(&mw, dW, plan));
             ANPD_TRY(make_tmap_bf16(&mh, dhi, rows, K, NB, false));
             ANPD_TRY(make_tmap_bf16(&ml, dlo, rows, K, NB, false));
             ANPD_TRY(gemm_tc_enqueue(plan, mw, mh, ml, rows, NB, dpart, (size_t)rows * N, N, derr, 0, nullptr));

@@ -575,17 +575,17 @@ __global__ void __launch_bounds__(256) accept_kernel(SeqState* seqs, const float
 //   part[0][row][n] = sum_k W[n][k] * (a_hi[row][k] + a_lo[row][k])
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict__ W, const bf16* __restrict__ a_hi,
-                                                         const bf16* __restrict__ a_lo, int rows, int N, int K,
+                                                         const bf16* __restrict__ a_lo, int rows, int N, int K, long long total, int G,
                                                          float* __restrict__ part, int ld_part) {
     const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (n >= N) return;
-    // tiled storage: tile (n / 128, k / 64) is 128 x 64 contiguous
+    // block storage: logical block (n / 128, k / 64) is 128 x 64 contiguous at its slot
     const int k_blocks = (K + 63) / 64;
-    const bf16* w = W + ((size_t)(n >> 7) * k_blocks * 128 + (n & 127)) * 64;
     for (int r0 = 0; r0 < rows; r0 += 8) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int k0 = lane * 8; k0 < K; k0 += 256) {
-            const uint4 wv = *(const uint4*)(w + (size_t)(k0 >> 6) * (128 * 64) + (k0 & 63));
+            const long long slot = gemm_block_slot((long long)(n >> 7) * k_blocks + (k0 >> 6), total, G);
+            const uint4 wv = *(const uint4*)(W + ((size_t)slot * 128 + (n & 127)) * 64 + (k0 & 63));
             const bf16* w8 = (const bf16*)&wv;
             float wf[8];
 #pragma unroll
@@ -627,7 +627,7 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
     if (kind == GK_DOWN) { a_hi = ws.act_hi; a_lo = ws.act_lo; maps = ws.map_act[mode]; }
     if (m->plain_gemm) {
         *seg_count_out = m->d_ones;
-        return gemm_plain_enqueue(W, a_hi, a_lo, rows, plan.N, plan.K, ws.part, ws.n_max_out, m->stream, &m->prof);
+        return gemm_plain_enqueue(plan, W, a_hi, a_lo, rows, ws.part, ws.n_max_out, m->stream, &m->prof);
     }
     const CUtensorMap& mw = kind == GK_LM ? m->map_lm : m->layers[layer].map[kind];
     ANPD_TRY(gemm_tc_enqueue(plan, mw, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)ws.r_max * ws.n_max_out,
@@ -663,10 +663,11 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
 
 }  // namespace
 
-anpd_status gemm_plain_enqueue(const bf16* W, const bf16* a_hi, const bf16* a_lo, int rows, int N, int K, float* part, int ld_part,
+anpd_status gemm_plain_enqueue(const GemmPlan& p, const bf16* W, const bf16* a_hi, const bf16* a_lo, int rows, float* part, int ld_part,
                                cudaStream_t st, Profiler* prof) {
-    LAUNCH(prof, st, KC_GEMM, 2.0 * (double)N * (double)K,
-           (gemm_rows8_kernel<<<(N + 7) / 8, 256, 0, st>>>(W, a_hi, a_lo, rows, N, K, part, ld_part)));
+    LAUNCH(prof, st, KC_GEMM, 2.0 * (double)p.N * (double)p.K,
+           (gemm_rows8_kernel<<<(p.N + 7) / 8, 256, 0, st>>>(W, a_hi, a_lo, rows, p.N, p.K, (long long)p.m_tiles * p.k_blocks, p.grid,
+                                                           part, ld_part)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }

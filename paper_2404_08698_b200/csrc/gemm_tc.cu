@@ -123,7 +123,7 @@ struct GemmArgs {
     int NB;                 // MMA N: rows padded to a multiple of 16
     int m_tiles, k_blocks;
     int stages;
-    int tmem_cols;          // power of two >= 2 * NB, >= 32
+    int tmem_cols;          // power of two >= 4 * NB (two accumulators of 2 * NB columns: W x hi and W x lo side by side)
     const int* first_cta;   // [m_tiles] CTA that owns the first k-block of a tile
     int* err;
 };
@@ -176,7 +176,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (!ok) break;
                 unsigned char* sa = smem + (size_t)stage * stage_bytes;
                 mbar_expect_tx(&bar_full[stage], (uint32_t)stage_bytes);
-                tma_load_2d(sa, &map_w, 0, (int)(blk * TILE_M), &bar_full[stage], pol_w);       // tile (tile, kb): 16 KB contiguous
+                tma_load_2d(sa, &map_w, 0, (int)(((blk - lo) * gridDim.x + blockIdx.x) * TILE_M), &bar_full[stage], pol_w);   // this CTA's slot of the step's window
                 tma_load_2d(sa + A_BYTES, &map_hi, kb * TILE_K, 0, &bar_full[stage], pol_a);
                 tma_load_2d(sa + A_BYTES + g.NB * 128, &map_lo, kb * TILE_K, 0, &bar_full[stage], pol_a);
                 ++issued;
@@ -196,7 +196,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.NB >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+            // fp32 accumulate, bf16 x bf16, both operands K-major, N = 2 * NB (hi rows then lo rows), M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * g.NB) >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
             int stage = 0;
             uint32_t phase = 0;
             int seg = 0;
@@ -209,20 +210,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 ok = mbar_wait(&bar_acc_empty[buf], (uint32_t)(((seg >> 1) & 1) ^ 1), abortp);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * g.NB);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * g.NB);
                 uint32_t acc = 0;
                 for (; blk < seg_end; ++blk) {
                     ok = mbar_wait(&bar_full[stage], phase, abortp);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + (size_t)stage * stage_bytes);
-                    const uint64_t da = make_smem_desc(sa), dh = make_smem_desc(sa + A_BYTES), dl = make_smem_desc(sa + A_BYTES + g.NB * 128);
+                    // the lo rows follow the hi rows in the stage, so one descriptor spans both: one MMA reads the
+                    // weight slice from shared memory once and yields W x hi in columns [0, NB) and W x lo in [NB, 2 NB)
+                    const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sa + A_BYTES);
 #pragma unroll
                     for (int k16 = 0; k16 < TILE_K / 16; ++k16) {
                         const uint64_t adv = (uint64_t)(k16 * 32 >> 4);     // 16 bf16 = 32 bytes along K inside the swizzle row
-                        tc_mma_bf16(d_tmem, da + adv, dh + adv, idesc, acc);
+                        tc_mma_bf16(d_tmem, da + adv, db + adv, idesc, acc);
                         acc = 1;
-                        tc_mma_bf16(d_tmem, da + adv, dl + adv, idesc, 1u);
                     }
                     tc_commit(&bar_empty[stage]);        // frees the stage once these MMAs have read it
                     if (++stage == g.stages) { stage = 0; phase ^= 1u; }
@@ -249,12 +251,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int n = tile * TILE_M + quad * 32 + lane;
             float* out = g.part + (size_t)ordinal * g.seg_stride + n;
             for (int c0 = 0; c0 < g.NB; c0 += 16) {
-                float v[16];
-                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * g.NB + c0), v);
+                float v[16], w[16];
+                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 2 * g.NB + c0), v);
+                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 2 * g.NB + g.NB + c0), w);
                 if (n < g.N) {
 #pragma unroll
                     for (int r = 0; r < 16; ++r)
-                        if (c0 + r < g.rows) out[(size_t)(c0 + r) * g.ld_part] = v[r];
+                        if (c0 + r < g.rows) out[(size_t)(c0 + r) * g.ld_part] = v[r] + w[r];
                 }
             }
             tc_fence_before();
@@ -276,12 +279,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 }
 
 template <typename T>
-__global__ void retile_kernel(const T* __restrict__ src, int rows, int K, int row_off, int k_blocks, bf16* __restrict__ dst) {
+__global__ void retile_kernel(const T* __restrict__ src, int rows, int K, int row_off, int k_blocks, long long total, int G,
+                              bf16* __restrict__ dst) {
     const int chunks = K / 8;                                  // 8 consecutive inputs never straddle a 64-wide block
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)rows * chunks; i += (size_t)gridDim.x * blockDim.x) {
         const int r = (int)(i / chunks), k0 = (int)(i % chunks) * 8;
         const int n = row_off + r;
-        bf16* out = dst + ((((size_t)(n >> 7) * k_blocks + (k0 >> 6)) * TILE_M + (n & 127)) * TILE_K + (k0 & 63));
+        const long long slot = gemm_block_slot((long long)(n >> 7) * k_blocks + (k0 >> 6), total, G);
+        bf16* out = dst + (((size_t)slot * TILE_M + (n & 127)) * TILE_K + (k0 & 63));
         const T* in = src + (size_t)r * K + k0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) out[e] = (bf16)in[e];
@@ -324,21 +329,18 @@ anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, 
     return ANPD_OK;
 }
 
-size_t gemm_tiled_elems(int N, int K) {
-    return (size_t)((N + TILE_M - 1) / TILE_M) * ((K + TILE_K - 1) / TILE_K) * TILE_M * TILE_K;
+size_t gemm_tiled_elems(const GemmPlan& p) { return (size_t)p.max_count * p.grid * TILE_M * TILE_K; }
+
+anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, const GemmPlan& p) {
+    return make_tmap_bf16(out, base_tiled, p.max_count * p.grid * TILE_M, TILE_K, TILE_M, true);
 }
 
-anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, int N, int K) {
-    const int rows = (int)(gemm_tiled_elems(N, K) / TILE_K);
-    return make_tmap_bf16(out, base_tiled, rows, TILE_K, TILE_M, true);
-}
-
-anpd_status gemm_retile_enqueue(const void* src, bool src_is_f32, int rows, int K, int row_off, bf16* dst_tiled, cudaStream_t st) {
-    const int k_blocks = (K + TILE_K - 1) / TILE_K;
-    const size_t work = (size_t)rows * (K / 8);
+anpd_status gemm_retile_enqueue(const GemmPlan& p, const void* src, bool src_is_f32, int rows, int row_off, bf16* dst_tiled, cudaStream_t st) {
+    const size_t work = (size_t)rows * (p.K / 8);
     const int blocks = (int)std::min<size_t>((work + 255) / 256, 148 * 16);
-    if (src_is_f32) retile_kernel<float><<<blocks, 256, 0, st>>>((const float*)src, rows, K, row_off, k_blocks, dst_tiled);
-    else retile_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)src, rows, K, row_off, k_blocks, dst_tiled);
+    const long long total = (long long)p.m_tiles * p.k_blocks;
+    if (src_is_f32) retile_kernel<float><<<blocks, 256, 0, st>>>((const float*)src, rows, p.K, row_off, p.k_blocks, total, p.grid, dst_tiled);
+    else retile_kernel<bf16><<<blocks, 256, 0, st>>>((const bf16*)src, rows, p.K, row_off, p.k_blocks, total, p.grid, dst_tiled);
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
@@ -351,6 +353,7 @@ void gemm_make_plan(GemmPlan* p, int N, int K, int num_sms) {
     p->k_blocks = (K + TILE_K - 1) / TILE_K;
     const long long total = (long long)p->m_tiles * p->k_blocks;
     p->grid = (int)std::min<long long>(num_sms, total);
+    p->max_count = (int)((total + p->grid - 1) / p->grid);
     p->first_cta.assign(p->m_tiles, 0);
     p->seg_count.assign(p->m_tiles, 0);
     p->max_segs = 0;
@@ -387,7 +390,7 @@ anpd_status gemm_tc_enqueue(const GemmPlan& plan, const CUtensorMap& map_w, cons
     g.m_tiles = plan.m_tiles; g.k_blocks = plan.k_blocks;
     const int smem = gemm_smem_bytes(NB, &g.stages);
     int cols = 32;
-    while (cols < 2 * NB) cols <<= 1;
+    while (cols < 4 * NB) cols <<= 1;
     g.tmem_cols = cols;
     g.first_cta = plan.d_first_cta;
     g.err = err;

@@ -135,6 +135,7 @@ constexpr int PREFILL_ROWS = 64;      // rows per prefill pass
 // each of which leaves one partial sum; consumers add them in that order.
 struct GemmPlan {
     int N, K, m_tiles, k_blocks, grid, max_segs;
+    int max_count;                    // most (tile, k-block) blocks any CTA owns
     std::vector<int> first_cta, seg_count;
     int* d_first_cta;
     int* d_seg_count;
@@ -233,16 +234,23 @@ anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev*
 
 // gemm_tc.cu
 anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, int box_rows, bool streamed);
-// Weight matrices are stored as a sequence of 128 x 64 tiles, tile (t, kb) at element ((t * k_blocks + kb) * 128) * 64.
-size_t gemm_tiled_elems(int N, int K);
-anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, int N, int K);
-// Scatters rows [row_off, row_off + rows) of a row-major [rows][K] source (bf16, or fp32 rounded to
-// bf16) into the tiled storage of a matrix with K inputs.  The padding must already be zero.
-anpd_status gemm_retile_enqueue(const void* src, bool src_is_f32, int rows, int K, int row_off, __nv_bfloat16* dst_tiled, cudaStream_t st);
+// Weight matrices are stored as 128 x 64 blocks of 16 KB.  The GEMM's CTA c owns the logical blocks
+// [c * total / G, (c + 1) * total / G) (logical index = tile * k_blocks + k_block) and reads its i-th
+// block at step i; that block is stored in slot i * G + c.  So at every step the G CTAs together read
+// one contiguous window of G * 16 KB, and the window sweeps through memory like a plain copy would.
+__host__ __device__ inline long long gemm_block_slot(long long logical, long long total, int G) {
+    const long long c = ((logical + 1) * G + total - 1) / total - 1;      // owner: largest c with c * total / G <= logical
+    return (logical - c * total / G) * G + c;
+}
 void gemm_make_plan(GemmPlan* p, int N, int K, int num_sms);
+size_t gemm_tiled_elems(const GemmPlan& p);
+anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, const GemmPlan& p);
+// Scatters rows [row_off, row_off + rows) of a row-major [rows][K] source (bf16, or fp32 rounded to
+// bf16) into the block storage of the plan's matrix.  The padding must already be zero.
+anpd_status gemm_retile_enqueue(const GemmPlan& p, const void* src, bool src_is_f32, int rows, int row_off, __nv_bfloat16* dst_tiled, cudaStream_t st);
 anpd_status gemm_tc_enqueue(const GemmPlan& plan, const CUtensorMap& map_w, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
                             int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,
                             Profiler* prof);
 // forward.cu: the plain (one warp per output feature) GEMM, kept as a cross-check
-anpd_status gemm_plain_enqueue(const __nv_bfloat16* W, const __nv_bfloat16* a_hi, const __nv_bfloat16* a_lo, int rows, int N, int K,
+anpd_status gemm_plain_enqueue(const GemmPlan& p, const __nv_bfloat16* W, const __nv_bfloat16* a_hi, const __nv_bfloat16* a_lo, int rows,
                                float* part, int ld_part, cudaStream_t st, Profiler* prof);
