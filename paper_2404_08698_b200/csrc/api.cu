@@ -11,6 +11,7 @@
 typedef __nv_bfloat16 bf16;
 
 long long g_launch_count = 0;
+bool g_use_pdl = std::getenv("ANPD_NO_PDL") == nullptr;
 static char g_last_error[256] = "";
 
 void anpd_note_cuda_error(cudaError_t e, const char* file, int line) {
@@ -59,6 +60,8 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restri
 }
 __global__ void set_int_kernel(int* p, int v) { *p = v; }
 __global__ void greedy_stage_kernel(SeqState* seqs) {
+    pdl_trigger();
+    pdl_wait();
     SeqState& s = seqs[blockIdx.x];
     s.last_tok = s.next_tok;
     s.draft_len = 0;
@@ -325,7 +328,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&ws.ao_hi, R * m->dq * 2}, {(void**)&ws.ao_lo, R * m->dq * 2},
         {(void**)&ws.act_hi, R * F * 2}, {(void**)&ws.act_lo, R * F * 2},
         {(void**)&ws.part, (size_t)ws.splits_max * R * ws.n_max_out * 4},
-        {(void**)&ws.q, R * m->dq * 4},
+        {(void**)&ws.q_hi, R * m->dq * 2}, {(void**)&ws.q_lo, R * m->dq * 2},
         {(void**)&ws.attn_m, n_part * 4}, {(void**)&ws.attn_l, n_part * 4}, {(void**)&ws.attn_o, n_part * hd * 4},
         {(void**)&ws.logits, R * V * 4},
         {(void**)&ws.amax_val, R * ws.amax_blocks * 4}, {(void**)&ws.amax_idx, R * ws.amax_blocks * 4},
@@ -525,7 +528,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
     cudaStream_t st = m->stream;
     auto enqueue = [&]() -> anpd_status {
         if (K > 0) ANPD_TRY(ngram_enqueue_step(d_ctxs, kv->seq, kv->batch, K, st, &m->prof));
-        else if (K == 0) { LAUNCH(&m->prof, st, KC_OTHER, 0, (greedy_stage_kernel<<<kv->batch, 1, 0, st>>>(kv->seq))); }
+        else if (K == 0) { LAUNCH(&m->prof, st, KC_OTHER, 0, (launch_k(greedy_stage_kernel, kv->batch, 1, 0, st, kv->seq))); }
         ANPD_TRY(plan_decode_enqueue(m, kv));
         ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
         ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
@@ -533,7 +536,11 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
     };
     if (m->prof.on || !kv->use_graphs || !kv->warm) {
         kv->warm = true;
-        return enqueue();
+        const bool pdl = g_use_pdl;
+        if (m->prof.on) g_use_pdl = false;            // per-launch timing needs kernels that do not overlap
+        const anpd_status rc = enqueue();
+        g_use_pdl = pdl;
+        return rc;
     }
     const uint64_t key = (uint64_t)(max_pos / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)mode << 24) |
                          ((uint64_t)(want_logits ? 1 : 0) << 28) | ((uint64_t)(d_ctxs ? 1 : 0) << 29);

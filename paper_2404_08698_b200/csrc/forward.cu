@@ -40,6 +40,8 @@ __device__ __forceinline__ float block_sum_256(float v, float* red /*[8]*/) {
 // ---------------------------------------------------------------------------------------------
 __global__ void plan_decode_kernel(SeqState* seqs, int* row_tok, int* row_pos, int* row_seq, int* row_ok,
                                    int vocab, int max_len) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int b = i / ANPD_ROWS, r = i % ANPD_ROWS;
     SeqState& s = seqs[b];
@@ -56,6 +58,8 @@ __global__ void plan_decode_kernel(SeqState* seqs, int* row_tok, int* row_pos, i
 __global__ void plan_prefill_kernel(const int* prompt, int seq, int start, int prompt_len, int rows,
                                     int* row_tok, int* row_pos, int* row_seq, int* row_ok, int vocab, int max_len,
                                     SeqState* seqs) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= rows) return;
     const int p = start + i;
@@ -96,6 +100,8 @@ __device__ __forceinline__ void store_split4(const float4 v, bf16* hi_ptr, bf16*
 __global__ void __launch_bounds__(NORM_THREADS) embed_norm_kernel(const bf16* __restrict__ embed, const int* __restrict__ row_tok,
                                                                   const float* __restrict__ gain, float eps, int d,
                                                                   float* __restrict__ x, bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[32];
     const int row = blockIdx.x, chunks = d >> 2;
     const bf16* e = embed + (size_t)row_tok[row] * d;
@@ -130,6 +136,8 @@ __global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restr
                                                                   const int* __restrict__ seg_count, size_t split_stride, int ld_part,
                                                                   const float* __restrict__ gain, float eps, int d,
                                                                   bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[32];
     const int row = blockIdx.x, chunks = d >> 2;
     float4 v[NORM_MAX_CHUNKS];
@@ -175,8 +183,10 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
                                        const int* __restrict__ row_pos, const int* __restrict__ row_seq,
                                        const int* __restrict__ row_ok, const float* __restrict__ rope_cos,
                                        const float* __restrict__ rope_sin, const int* __restrict__ page_table,
-                                       int pages_per_seq, int Hq, int Hkv, int hd, float* __restrict__ q,
-                                       bf16* __restrict__ kpool_l, bf16* __restrict__ vpool_l) {
+                                       int pages_per_seq, int Hq, int Hkv, int hd, float q_scale, bf16* __restrict__ q_hi,
+                                       bf16* __restrict__ q_lo, bf16* __restrict__ kpool_l, bf16* __restrict__ vpool_l) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
     const float* pr = part + (size_t)row * ld_part + (size_t)head * hd;
     float a = 0.0f, b = 0.0f;
@@ -189,8 +199,11 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
         a = ra; b = rb;
     }
     if (head < Hq) {
-        q[(size_t)row * Hq * hd + head * hd + i] = a;
-        q[(size_t)row * Hq * hd + head * hd + i + half] = b;
+        // queries leave as two bf16 terms, already multiplied by log2(e) / sqrt(hd): the attention kernel
+        // takes them as MMA fragments and works with base-2 exponentials
+        const size_t o = (size_t)row * Hq * hd + head * hd + i;
+        split_bf16(a * q_scale, q_hi[o], q_lo[o]);
+        split_bf16(b * q_scale, q_hi[o + half], q_lo[o + half]);
         return;
     }
     if (!row_ok[row]) return;
@@ -246,11 +259,14 @@ constexpr int ATTN_THREADS = 128;
 constexpr int KEY_BLOCK = 32;
 
 template <int HD>
-__global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float* __restrict__ q, const bf16* __restrict__ kpool_l,
-                                                                    const bf16* __restrict__ vtpool_l, const int* __restrict__ page_table,
-                                                                    int pages_per_seq, const int* __restrict__ row_pos,
-                                                                    const int* __restrict__ row_seq, int Hq, int Hkv, float scale,
-                                                                    float* __restrict__ pm, float* __restrict__ pl, float* __restrict__ po) {
+__global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const bf16* __restrict__ q_hi, const bf16* __restrict__ q_lo,
+                                                                    const bf16* __restrict__ kpool_l, const bf16* __restrict__ vtpool_l,
+                                                                    const int* __restrict__ page_table, int pages_per_seq,
+                                                                    const int* __restrict__ row_pos, const int* __restrict__ row_seq, int Hq,
+                                                                    int Hkv, float* __restrict__ pm, float* __restrict__ pl,
+                                                                    float* __restrict__ po) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int SLABS = HD / 32;            // 32-wide slabs of the head dimension (two MMAs each)
     constexpr int DT = HD / 8;                // 8-wide tiles of the head dimension for P V
     constexpr int OP = HD + 4;                // padded row of the merge buffer
@@ -260,7 +276,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
     unsigned char* Ks = attn_smem;                                  // [KV_PAGE][KPITCH]
     unsigned char* Vs = attn_smem + KV_PAGE * KPITCH;               // [HD][VPITCH]
     float (*sm_o)[16][OP] = (float (*)[16][OP])Ks;                  // [4][16][OP], reuses the K staging area after the last MMA
-    __shared__ float sm_m[4][16], sm_l[4][16];
+    __shared__ float sm_m[4][16], sm_l[4][16], sm_w[4][16];
 
     const int G = Hq / Hkv;
     const int MT = (ANPD_ROWS * G + 15) / 16;             // 16-row tiles of query vectors: 1, 1, 2, 4 for G = 1, 2, 4, 8
@@ -301,17 +317,15 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
         const bool valid = qi < ANPD_ROWS * G;
         const int r = valid ? qi / G : 0, hl = valid ? qi % G : 0;
         qpos[h] = valid ? pos_lo + r : -1;                // -1: padding row, sees no key
-        const float* qp = q + (size_t)(r0 + r) * Hq * HD + (size_t)(kvh * G + hl) * HD + 8 * t;
+        const size_t qoff = (size_t)(r0 + r) * Hq * HD + (size_t)(kvh * G + hl) * HD + 8 * t;
 #pragma unroll
         for (int s = 0; s < SLABS; ++s) {
-            float4 f0 = make_float4(0.f, 0.f, 0.f, 0.f), f1 = f0;
-            if (valid) { f0 = *(const float4*)(qp + 32 * s); f1 = *(const float4*)(qp + 32 * s + 4); }
-            // first MMA of the slab: elements 0..3; second: elements 4..7.  Register h holds row gid + 8h
-            // for logical k = 2t, 2t+1; register 2 + h the same row for logical k = 2t+8, 2t+9.
-            qh[s][0][h] = pack_split(f0.x * scale, f0.y * scale, ql[s][0][h]);
-            qh[s][0][2 + h] = pack_split(f0.z * scale, f0.w * scale, ql[s][0][2 + h]);
-            qh[s][1][h] = pack_split(f1.x * scale, f1.y * scale, ql[s][1][h]);
-            qh[s][1][2 + h] = pack_split(f1.z * scale, f1.w * scale, ql[s][1][2 + h]);
+            // 16 bytes = elements 8t..8t+7 of the slab: (e0,e1),(e2,e3) feed the slab's first MMA, (e4,e5),(e6,e7)
+            // the second.  Register h holds row gid + 8h for logical k = 2t, 2t+1; register 2 + h for 2t+8, 2t+9.
+            uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+            if (valid) { a = *(const uint4*)(q_hi + qoff + 32 * s); b = *(const uint4*)(q_lo + qoff + 32 * s); }
+            qh[s][0][h] = a.x; qh[s][0][2 + h] = a.y; qh[s][1][h] = a.z; qh[s][1][2 + h] = a.w;
+            ql[s][0][h] = b.x; ql[s][0][2 + h] = b.y; ql[s][1][h] = b.z; ql[s][1][2 + h] = b.w;
         }
     }
 
@@ -358,13 +372,13 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
             const float m_new = fmaxf(m_run[h], mx);
             const bool none = (m_new == -CUDART_INF_F);
-            const float resc = none ? 1.0f : expf(m_run[h] - m_new);
+            const float resc = none ? 1.0f : exp2f(m_run[h] - m_new);
             float psum = 0.0f;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const float p = none ? 0.0f : expf(sc[j][2 * h + e] - m_new);
+                    const float p = none ? 0.0f : exp2f(sc[j][2 * h + e] - m_new);
                     sc[j][2 * h + e] = p;
                     psum += p;
                 }
@@ -409,23 +423,38 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
         sm_o[warp][gid + 8][8 * d + 2 * t + 1] = o[d][3];
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < MT * 16 * HD; idx += ATTN_THREADS) {
-        const int dim = idx % HD, rowi = (idx / HD) % 16, tile = idx / (HD * 16);
-        const int qi = tile * 16 + rowi;
-        if (qi >= ANPD_ROWS * G) continue;
+    // weights of the merged warps, once per query vector
+    if (threadIdx.x < MT * 16) {
+        const int tile = threadIdx.x / 16, rowi = threadIdx.x % 16;
         float M = -CUDART_INF_F;
         for (int k = 0; k < KG; ++k) M = fmaxf(M, sm_m[k * MT + tile][rowi]);
-        float L = 0.0f, O = 0.0f;
+        float L = 0.0f;
         for (int k = 0; k < KG; ++k) {
             const float mk = sm_m[k * MT + tile][rowi];
-            const float w = (mk == -CUDART_INF_F) ? 0.0f : expf(mk - M);
+            const float w = (mk == -CUDART_INF_F) ? 0.0f : exp2f(mk - M);
+            sm_w[k * MT + tile][rowi] = w;
             L = fmaf(sm_l[k * MT + tile][rowi], w, L);
-            O = fmaf(sm_o[k * MT + tile][rowi][dim], w, O);
         }
-        const int r = qi / G, hl = qi % G;
-        const size_t out = ((size_t)(r0 + r) * Hq + (kvh * G + hl)) * pages_per_seq + c;
-        po[out * HD + dim] = O;
-        if (dim == 0) { pm[out] = M; pl[out] = L; }
+        const int qi = tile * 16 + rowi;
+        if (qi < ANPD_ROWS * G) {
+            const size_t out = ((size_t)(r0 + qi / G) * Hq + (kvh * G + qi % G)) * pages_per_seq + c;
+            pm[out] = M;
+            pl[out] = L;
+        }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < MT * 16 * (HD / 4); idx += ATTN_THREADS) {
+        const int d4 = idx % (HD / 4), rowi = (idx / (HD / 4)) % 16, tile = idx / ((HD / 4) * 16);
+        const int qi = tile * 16 + rowi;
+        if (qi >= ANPD_ROWS * G) continue;
+        float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = 0; k < KG; ++k) {
+            const float w = sm_w[k * MT + tile][rowi];
+            const float4 v = *(const float4*)&sm_o[k * MT + tile][rowi][4 * d4];
+            O.x = fmaf(v.x, w, O.x); O.y = fmaf(v.y, w, O.y); O.z = fmaf(v.z, w, O.z); O.w = fmaf(v.w, w, O.w);
+        }
+        const size_t out = ((size_t)(r0 + qi / G) * Hq + (kvh * G + qi % G)) * pages_per_seq + c;
+        *(float4*)(po + out * HD + 4 * d4) = O;
     }
 }
 
@@ -433,6 +462,8 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const float*
 __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* __restrict__ pl, const float* __restrict__ po,
                                     const int* __restrict__ row_pos, int Hq, int hd, int pages_per_seq,
                                     bf16* __restrict__ ao_hi, bf16* __restrict__ ao_lo) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x, head = blockIdx.y, dim = threadIdx.x;
     const int nc = row_pos[row] / KV_PAGE + 1;
     const size_t base = ((size_t)row * Hq + head) * pages_per_seq;
@@ -440,7 +471,7 @@ __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* _
     for (int c = 0; c < nc; ++c) M = fmaxf(M, pm[base + c]);
     float L = 0.0f, o = 0.0f;
     for (int c = 0; c < nc; ++c) {
-        const float w = expf(pm[base + c] - M);
+        const float w = exp2f(pm[base + c] - M);            // partial maxima are in the base-2 domain
         L = fmaf(pl[base + c], w, L);
         o = fmaf(po[(base + c) * hd + dim], w, o);
     }
@@ -456,6 +487,8 @@ __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* _
 // ---------------------------------------------------------------------------------------------
 __global__ void swiglu_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride, int ld_part, int F,
                               bf16* __restrict__ act_hi, bf16* __restrict__ act_lo) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= F) return;
     const float* pr = part + (size_t)row * ld_part;
@@ -477,6 +510,8 @@ constexpr int AMAX_COLS = 1024;
 __global__ void __launch_bounds__(256) argmax_partial_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride,
                                                              int ld_part, int V, float* __restrict__ logits,
                                                              float* __restrict__ amax_val, int* __restrict__ amax_idx, int nblk) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float sv[8];
     __shared__ int si[8];
     const int row = blockIdx.y;
@@ -512,6 +547,8 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const float* __rest
 __global__ void __launch_bounds__(256) accept_kernel(SeqState* seqs, const float* __restrict__ amax_val,
                                                      const int* __restrict__ amax_idx, int nblk, int mode,
                                                      const NgramDev* ctxs, int seq_arg, int last_row, int prompt_len) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ int pred[ANPD_ROWS];
     const int b = (mode == ACCEPT_PREFILL) ? seq_arg : blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -577,6 +614,8 @@ __global__ void __launch_bounds__(256) accept_kernel(SeqState* seqs, const float
 __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict__ W, const bf16* __restrict__ a_hi,
                                                          const bf16* __restrict__ a_lo, int rows, int N, int K, long long total, int G,
                                                          float* __restrict__ part, int ld_part) {
+    pdl_trigger();
+    pdl_wait();
     const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (n >= N) return;
     // block storage: logical block (n / 128, k / 64) is 128 x 64 contiguous at its slot
@@ -651,12 +690,12 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     }
     dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (attn_partial_kernel<HD><<<grid, ATTN_THREADS, smem, m->stream>>>(ws.q, kv->kpool + layer * layer_elems, kv->vpool + layer * layer_elems,
-                                                                            kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq,
-                                                                            c.n_q_heads, c.n_kv_heads, 1.0f / sqrtf((float)HD),
-                                                                            ws.attn_m, ws.attn_l, ws.attn_o)));
+           (launch_k(attn_partial_kernel<HD>, grid, ATTN_THREADS, smem, m->stream, ws.q_hi, ws.q_lo, kv->kpool + layer * layer_elems,
+                                                                            kv->vpool + layer * layer_elems, kv->page_table, kv->pages_per_seq,
+                                                                            ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, ws.attn_m,
+                                                                            ws.attn_l, ws.attn_o)));
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (attn_combine_kernel<<<dim3(rows, c.n_q_heads), HD, 0, m->stream>>>(ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
+           (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
     return ANPD_OK;
 }
@@ -666,7 +705,7 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
 anpd_status gemm_plain_enqueue(const GemmPlan& p, const bf16* W, const bf16* a_hi, const bf16* a_lo, int rows, float* part, int ld_part,
                                cudaStream_t st, Profiler* prof) {
     LAUNCH(prof, st, KC_GEMM, 2.0 * (double)p.N * (double)p.K,
-           (gemm_rows8_kernel<<<(p.N + 7) / 8, 256, 0, st>>>(W, a_hi, a_lo, rows, p.N, p.K, (long long)p.m_tiles * p.k_blocks, p.grid,
+           (launch_k(gemm_rows8_kernel, (p.N + 7) / 8, 256, 0, st, W, a_hi, a_lo, rows, p.N, p.K, (long long)p.m_tiles * p.k_blocks, p.grid,
                                                            part, ld_part)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
@@ -675,7 +714,7 @@ anpd_status gemm_plain_enqueue(const GemmPlan& p, const bf16* W, const bf16* a_h
 anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv) {
     Workspace& ws = kv->ws;
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
-           (plan_decode_kernel<<<kv->batch, ANPD_ROWS, 0, m->stream>>>(kv->seq, ws.row_tok, ws.row_pos, ws.row_seq, ws.row_ok,
+           (launch_k(plan_decode_kernel, kv->batch, ANPD_ROWS, 0, m->stream, kv->seq, ws.row_tok, ws.row_pos, ws.row_seq, ws.row_ok,
                                                                       m->cfg.vocab, kv->max_len)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
@@ -684,7 +723,7 @@ anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv) {
 anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start, int prompt_len, int rows) {
     Workspace& ws = kv->ws;
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
-           (plan_prefill_kernel<<<(rows + 127) / 128, 128, 0, m->stream>>>(kv->d_prompt, seq, start, prompt_len, rows, ws.row_tok,
+           (launch_k(plan_prefill_kernel, (rows + 127) / 128, 128, 0, m->stream, kv->d_prompt, seq, start, prompt_len, rows, ws.row_tok,
                                                                           ws.row_pos, ws.row_seq, ws.row_ok, m->cfg.vocab,
                                                                           kv->max_len, kv->seq)));
     CUDA_TRY(cudaGetLastError());
@@ -695,7 +734,7 @@ anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev*
     Workspace& ws = kv->ws;
     const int blocks = (mode == ACCEPT_PREFILL) ? 1 : kv->batch;
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
-           (accept_kernel<<<blocks, 256, 0, m->stream>>>(kv->seq, ws.amax_val, ws.amax_idx, ws.amax_blocks, mode, d_ctxs, seq,
+           (launch_k(accept_kernel, blocks, 256, 0, m->stream, kv->seq, ws.amax_val, ws.amax_idx, ws.amax_blocks, mode, d_ctxs, seq,
                                                         last_row, prompt_len)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
@@ -711,36 +750,36 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * hd;
     const int* segs = nullptr;
 
-    LAUNCH(pf, st, KC_OTHER, 0, (embed_norm_kernel<<<rows, NORM_THREADS, 0, st>>>(m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
+    LAUNCH(pf, st, KC_OTHER, 0, (launch_k(embed_norm_kernel, rows, NORM_THREADS, 0, st, m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
                                                                       ws.x, ws.h_hi, ws.h_lo)));
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& w = m->layers[l];
         ANPD_TRY(gemm_enqueue(m, kv, GK_QKV, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (qkv_rope_append_kernel<<<dim3(rows, c.n_q_heads + 2 * c.n_kv_heads), hd / 2, 0, st>>>(
+               (launch_k(qkv_rope_append_kernel, dim3(rows, c.n_q_heads + 2 * c.n_kv_heads), hd / 2, 0, st, 
                    ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
-                   kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, hd, ws.q, kv->kpool + l * layer_elems,
-                   kv->vpool + l * layer_elems)));
+                   kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, hd, 1.4426950408889634f / sqrtf((float)hd), ws.q_hi,
+                   ws.q_lo, kv->kpool + l * layer_elems, kv->vpool + l * layer_elems)));
         if (hd == 128) ANPD_TRY(attn_enqueue<128>(m, kv, l, rows, max_pos));
         else ANPD_TRY(attn_enqueue<64>(m, kv, l, rows, max_pos));
         ANPD_TRY(gemm_enqueue(m, kv, GK_O, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (resid_norm_kernel<<<rows, NORM_THREADS, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
+               (launch_k(resid_norm_kernel, rows, NORM_THREADS, 0, st, ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
         ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (swiglu_kernel<<<dim3((F + 255) / 256, rows), 256, 0, st>>>(ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
+               (launch_k(swiglu_kernel, dim3((F + 255) / 256, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
                                                                           ws.act_lo)));
         ANPD_TRY(gemm_enqueue(m, kv, GK_DOWN, l, rows, &segs));
         const float* next_gain = (l + 1 < c.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
         LAUNCH(pf, st, KC_OTHER, 0,
-               (resid_norm_kernel<<<rows, NORM_THREADS, 0, st>>>(ws.x, ws.part, segs, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
+               (launch_k(resid_norm_kernel, rows, NORM_THREADS, 0, st, ws.x, ws.part, segs, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
     }
     if (!head) { CUDA_TRY(cudaGetLastError()); return ANPD_OK; }
     ANPD_TRY(gemm_enqueue(m, kv, GK_LM, 0, rows, &segs));
     LAUNCH(pf, st, KC_OTHER, 0,
-           (argmax_partial_kernel<<<dim3(ws.amax_blocks, rows), 256, 0, st>>>(ws.part, segs, sstride, ws.n_max_out, V,
+           (launch_k(argmax_partial_kernel, dim3(ws.amax_blocks, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, V,
                                                                              want_logits ? ws.logits : nullptr, ws.amax_val,
                                                                              ws.amax_idx, ws.amax_blocks)));
     CUDA_TRY(cudaGetLastError());

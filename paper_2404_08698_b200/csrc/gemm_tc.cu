@@ -137,6 +137,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __shared__ int abort_flag;
 
     // the swizzled tiles need 1024-byte alignment in the shared address space
+    pdl_trigger();
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int stage_bytes = A_BYTES + 2 * g.NB * 128;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -170,8 +171,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            for (long long blk = lo; blk < hi && ok; ++blk) {
-                const int tile = (int)(blk / g.k_blocks), kb = (int)(blk % g.k_blocks);
+            // The weights do not depend on the previous kernel: request the first ring of weight tiles at
+            // once, and only then wait for the kernel that produces this GEMM's activations.
+            const long long ahead = min((long long)g.stages, hi - lo);
+            for (long long i = 0; i < ahead; ++i) {
+                unsigned char* sa = smem + (size_t)i * stage_bytes;
+                mbar_expect_tx(&bar_full[i], (uint32_t)stage_bytes);
+                tma_load_2d(sa, &map_w, 0, (int)((i * gridDim.x + blockIdx.x) * TILE_M), &bar_full[i], pol_w);
+            }
+            pdl_wait();
+            for (long long i = 0; i < ahead; ++i) {
+                unsigned char* sa = smem + (size_t)i * stage_bytes;
+                const int kb = (int)((lo + i) % g.k_blocks);
+                tma_load_2d(sa + A_BYTES, &map_hi, kb * TILE_K, 0, &bar_full[i], pol_a);
+                tma_load_2d(sa + A_BYTES + g.NB * 128, &map_lo, kb * TILE_K, 0, &bar_full[i], pol_a);
+            }
+            issued = ahead;
+            stage = (int)(ahead % g.stages);
+            phase = (ahead == g.stages) ? 1u : 0u;
+            for (long long blk = lo + ahead; blk < hi && ok; ++blk) {
+                const int kb = (int)(blk % g.k_blocks);
                 ok = mbar_wait(&bar_empty[stage], phase ^ 1u, abortp);
                 if (!ok) break;
                 unsigned char* sa = smem + (size_t)stage * stage_bytes;
@@ -195,6 +214,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
+        pdl_wait();
         if (lane == 0) {
             // fp32 accumulate, bf16 x bf16, both operands K-major, N = 2 * NB (hi rows then lo rows), M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * g.NB) >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
@@ -236,6 +256,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
     } else {
         // ---------------- epilogue: TMEM -> registers -> partial sums in global memory ----------------
+        pdl_wait();                                       // the partial-sum buffer may still be read by the previous kernel
         const int quad = warp & 3;                        // a warp may only touch TMEM lanes 32*(warp%4)..+31
         int seg = 0;
         bool ok = true;
@@ -395,7 +416,7 @@ anpd_status gemm_tc_enqueue(const GemmPlan& plan, const CUtensorMap& map_w, cons
     g.first_cta = plan.d_first_cta;
     g.err = err;
     LAUNCH(prof, st, KC_GEMM, 2.0 * (double)plan.N * (double)plan.K,
-           (gemm_tc_kernel<<<plan.grid, GEMM_THREADS, smem, st>>>(map_w, map_hi, map_lo, g)));
+           (launch_k(gemm_tc_kernel, plan.grid, GEMM_THREADS, smem, st, map_w, map_hi, map_lo, g)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }

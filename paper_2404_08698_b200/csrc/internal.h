@@ -64,6 +64,33 @@ extern long long g_launch_count;
     } while (0)
 
 // ---------------------------------------------------------------------------------------------
+// programmatic dependent launch
+// Every kernel of a step is launched so that it may start while its predecessor is still running:
+// it signals its own successor at once (pdl_trigger) and blocks in pdl_wait before it touches
+// anything an earlier kernel produced (or overwrites anything an earlier kernel may still read).
+// The weight-streaming GEMM uses the gap: its producer thread requests the first weight tiles before
+// it waits, so HBM keeps streaming through the small kernels between two GEMMs.  A kernel launched
+// without the attribute (or with ANPD_NO_PDL set) sees both calls as no-ops.
+// ---------------------------------------------------------------------------------------------
+extern bool g_use_pdl;
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_use_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
+// ---------------------------------------------------------------------------------------------
 // per-sequence step state (device)
 // ---------------------------------------------------------------------------------------------
 struct SeqState {
@@ -184,7 +211,7 @@ struct Workspace {
     __nv_bfloat16 *ao_hi, *ao_lo;     // [r_max, dq]  attention output, input of the O projection
     __nv_bfloat16 *act_hi, *act_lo;   // [r_max, F]   SwiGLU output, input of the down projection
     float* part;                      // [splits_max, r_max, n_max_out] GEMM partial sums
-    float* q;                         // [r_max, dq]
+    __nv_bfloat16 *q_hi, *q_lo;       // [r_max, dq] rotated queries x log2(e)/sqrt(hd), as two bf16 terms
     float *attn_m, *attn_l, *attn_o;  // per (row, q head, key chunk): max, sum, weighted values
     float* logits;                    // [r_max, V]
     float* amax_val; int* amax_idx;   // [r_max, amax_blocks]

@@ -123,6 +123,8 @@ __global__ void ngram_bulk_kernel(NgramDev c, int from, int to) {
 // draft K tokens by chained back-off queries.  Warp w of the first n_max-n_min+1 warps serves
 // level n_max - w, so the levels of one query are probed side by side and the longest wins.
 __global__ void __launch_bounds__(STEP_THREADS) ngram_step_kernel(const NgramDev* ctxs, SeqState* seqs, int K) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ NgramDev c;
     __shared__ int tail[ANPD_N_MAX - 1 + ANPD_K_MAX + 1];
     __shared__ int res[ANPD_N_MAX];
@@ -198,7 +200,7 @@ anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof
 
 anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batch, int K,
                                cudaStream_t st, Profiler* prof) {
-    LAUNCH(prof, st, KC_NGRAM, 0, (ngram_step_kernel<<<batch, STEP_THREADS, 0, st>>>(d_ctxs, d_seq, K)));
+    LAUNCH(prof, st, KC_NGRAM, 0, (launch_k(ngram_step_kernel, batch, STEP_THREADS, 0, st, d_ctxs, d_seq, K)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
