@@ -230,6 +230,24 @@ long long anpd_launch_count(int reset);
  * reference kernel the tensor-core kernel is cross-checked against. */
 anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a, int rows, float* out, int plain);
 
+/* The same product as anpd_debug_gemm for callers that must not allocate device memory; the paper
+ * has no counterpart for this call.  It exists for code that cannot afford a cudaMalloc inside the
+ * library: a serving loop that an allocation's device-wide synchronisation would stall, or a process
+ * whose device memory is wholly owned by another allocator, where a hidden allocation can fail.
+ * All buffers are the caller's and live on the current DEVICE: w_bf16_dev N*K bf16 bit patterns
+ * (row-major [N][K]), a_dev rows*K fp32, out_dev rows*N fp32 (written).  Work is issued on cuda_stream
+ * and the call returns after it has completed.  Every temporary lives in one fixed array of about
+ * 7 MiB that each GPU holds from the moment it loads the library until the process exits; the call
+ * never calls cudaMalloc, cudaFree or any allocating routine.
+ * Limits: rows a multiple of 8, at most 32; K a multiple of 8; ceil(N/128) * ceil(K/64) <= 128.
+ * Larger sizes return ANPD_ERR_CAPACITY (and say so on stderr) without touching anything.
+ * The array is shared by all calls on a device and keeps the previous call's contents; the call
+ * clears what must start at zero itself.  Calls that overlap on the GPU (two streams, two threads)
+ * race on it: issue them one after the other.  The first call on a device looks up the array's
+ * device address; make that first call before any stream capture begins. */
+anpd_status anpd_gemm_static(const uint16_t* w_bf16_dev, int N, int K, const float* a_dev, int rows,
+                             float* out_dev, void* cuda_stream);
+
 const char* anpd_status_string(anpd_status s);
 
 #ifdef __cplusplus

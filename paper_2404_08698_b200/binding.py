@@ -93,6 +93,7 @@ SIGNATURES = {
     "anpd_launch_count": (C.c_longlong, [C.c_int]),
     "anpd_debug_gemm": (C.c_int, [C.POINTER(C.c_uint16), C.c_int, C.c_int, C.POINTER(C.c_float), C.c_int,
                                   C.POINTER(C.c_float), C.c_int]),
+    "anpd_gemm_static": (C.c_int, [_P, C.c_int, C.c_int, _P, C.c_int, _P, _P]),
     "anpd_status_string": (C.c_char_p, [C.c_int]),
 }
 
@@ -343,3 +344,14 @@ def anpd_debug_gemm(w_bf16, a, plain: bool = False) -> np.ndarray:
     _check(lib().anpd_debug_gemm(wb.ctypes.data_as(C.POINTER(C.c_uint16)), N, K, a.ctypes.data_as(C.POINTER(C.c_float)), rows,
                                  out.ctypes.data_as(C.POINTER(C.c_float)), int(plain)), "anpd_debug_gemm")
     return out
+
+
+def anpd_gemm_static(w_bf16_dev, a_dev, out_dev, stream: int = 0) -> None:
+    """out_dev[rows, N] = a_dev[rows, K] @ w_bf16_dev[N, K]^T with no allocation inside the library.
+    All three are CUDA tensors owned by the caller (bf16, fp32, fp32); out_dev is overwritten."""
+    N, K = w_bf16_dev.shape
+    rows = a_dev.shape[0]
+    assert w_bf16_dev.is_cuda and a_dev.is_cuda and out_dev.is_cuda
+    assert w_bf16_dev.is_contiguous() and a_dev.is_contiguous() and out_dev.is_contiguous()
+    _check(lib().anpd_gemm_static(_P(w_bf16_dev.data_ptr()), N, K, _P(a_dev.data_ptr()), rows, _P(out_dev.data_ptr()),
+                                  _P(stream)), "anpd_gemm_static")
