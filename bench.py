@@ -201,6 +201,16 @@ def verify_microbench(args, A, wl, model, stream) -> None:
                       "rows": rows_out}))
 
 
+def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
+    """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
+    time.  `dist` is torch.distributed (or None for one process)."""
+    if dist is not None and world > 1:
+        t = torch.tensor([seconds], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        seconds = float(t.item())
+    return seconds, world * units_per_rank / seconds
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -291,11 +301,8 @@ def main() -> None:
     clocks = sampler.stop()
     launches = A.anpd_launch_count(True)
     anpd_tokens = out_dev.cpu().numpy().copy()
-    if dist is not None:
-        t = torch.tensor([t_anpd], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_anpd = float(t.item())
-    value = world * args.steps * wl.max_new / t_anpd
+    t_anpd_local = t_anpd
+    t_anpd, value = job_time_and_value(dist, t_anpd, args.steps * wl.max_new, world, "cuda")
 
     # ---- the same build's plain greedy decode --------------------------------------------------
     t_greedy, st_greedy = timed(0, args.steps, 1)
@@ -310,11 +317,8 @@ def main() -> None:
         out_host, _ = A.anpd_generate(model, kv, ctx, prompt, wl.max_new, wl.K)
     torch.cuda.synchronize()
     t_e2e = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([t_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_e2e = float(t.item())
-    e2e = {"value": world * args.steps * wl.max_new / t_e2e, "unit": UNIT,
+    t_e2e, e2e_value = job_time_and_value(dist, t_e2e, args.steps * wl.max_new, world, "cuda")
+    e2e = {"value": e2e_value, "unit": UNIT,
            "h2d_bytes_per_step": int(prompt.nbytes), "d2h_bytes_per_step": int(out_host.nbytes)}
 
     # ---- verify-step microbenchmark at the end-of-prompt KV length ------------------------------
@@ -367,7 +371,7 @@ def main() -> None:
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
         "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline,
-        "anpd": {"tokens_per_s": args.steps * wl.max_new / t_anpd if world == 1 else value / world,
+        "anpd": {"tokens_per_s": args.steps * wl.max_new / t_anpd_local,
                  "decode_tokens_per_s": st_anpd["generated"] / (st_anpd["ms_decode"] * 1e-3),
                  "ms_prefill": st_anpd["ms_prefill"], "ms_decode": st_anpd["ms_decode"], "steps": st_anpd["steps"],
                  "mean_accepted_per_step": st_anpd["accepted"] / max(st_anpd["steps"], 1),
@@ -375,7 +379,7 @@ def main() -> None:
                  "hist_accepted": st_anpd["hist_accepted"]},
         "greedy": {"tokens_per_s": greedy_tps, "decode_tokens_per_s": st_greedy["generated"] / (st_greedy["ms_decode"] * 1e-3),
                    "ms_prefill": st_greedy["ms_prefill"], "ms_decode": st_greedy["ms_decode"]},
-        "speedup_vs_greedy": (args.steps * wl.max_new / t_anpd) / greedy_tps if world == 1 else None,
+        "speedup_vs_greedy": (args.steps * wl.max_new / t_anpd_local) / greedy_tps,
         "decode_speedup_vs_greedy": st_greedy["ms_decode"] / st_anpd["ms_decode"] * st_anpd["generated"] / st_greedy["generated"],
         "anpd_equals_greedy": lossless,
         "verify_step": {"kv_len": P, "rows": A.ROWS, "ms": ms_verify, "bytes": step_bytes, "gbs": verify_gbs,

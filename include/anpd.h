@@ -124,7 +124,7 @@ anpd_status anpd_model_destroy(anpd_model* m);
 
 /* ---- KV cache ------------------------------------------------------------------------
  * Paged bf16 cache for `batch` independent sequences of at most max_len positions each
- * (max_len is rounded up to whole pages; a step needs kv_len + 8 <= max_len).  Also holds the
+ * (max_len <= 32768 is rounded up to whole pages, batch <= 16; a step needs kv_len + 8 <= max_len).  Also holds the
  * activation buffers of a forward, so a kv handle is tied to the model it was created for.
  * shuffle_pages != 0 permutes the physical page order (results must not change). */
 anpd_status anpd_kv_create(const anpd_model* m, int max_len, int batch, int shuffle_pages, anpd_kv** out);

@@ -294,7 +294,7 @@ anpd_status anpd_model_destroy(anpd_model* m) {
 // KV cache + workspace
 // ---------------------------------------------------------------------------------------------
 anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shuffle_pages, anpd_kv** out) {
-    if (!cm || !out || max_len < ANPD_ROWS || batch < 1 || batch > 16) return ANPD_ERR_ARG;
+    if (!cm || !out || max_len < ANPD_ROWS || max_len > 256 * KV_PAGE || batch < 1 || batch > 16) return ANPD_ERR_ARG;
     anpd_model* m = const_cast<anpd_model*>(cm);
     const anpd_model_config& c = m->cfg;
     anpd_kv* kv = new (std::nothrow) anpd_kv();

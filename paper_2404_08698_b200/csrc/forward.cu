@@ -458,28 +458,62 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const bf16* 
     }
 }
 
-// One block per (row, q head): fold the pages 0..pos/KV_PAGE in order, write the output as hi+lo.
+// One block per (row, q head): fold the pages 0..pos/KV_PAGE, write the output as hi+lo.  The block is
+// hd x 4 threads: thread (dim, k) adds the pages k, k+4, k+8, ... in ascending order, the four slices
+// are then added in slice order - a fixed order for a given number of pages.  Page maxima and sums are
+// fetched once by the first threads, so the kernel is about two memory round trips long.
+constexpr int COMBINE_SLICES = 4;
+constexpr int COMBINE_MAX_PAGES = 256;
 __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* __restrict__ pl, const float* __restrict__ po,
                                     const int* __restrict__ row_pos, int Hq, int hd, int pages_per_seq,
                                     bf16* __restrict__ ao_hi, bf16* __restrict__ ao_lo) {
     pdl_trigger();
     pdl_wait();
-    const int row = blockIdx.x, head = blockIdx.y, dim = threadIdx.x;
-    const int nc = row_pos[row] / KV_PAGE + 1;
+    __shared__ float s_w[COMBINE_MAX_PAGES];            // page maxima, then page weights
+    __shared__ float s_l[COMBINE_MAX_PAGES];
+    __shared__ float s_o[COMBINE_SLICES][128];
+    __shared__ float s_L;
+    const int row = blockIdx.x, head = blockIdx.y;
+    const int dim = threadIdx.x % hd, slice = threadIdx.x / hd;
+    const int nc = min(row_pos[row] / KV_PAGE + 1, COMBINE_MAX_PAGES);
     const size_t base = ((size_t)row * Hq + head) * pages_per_seq;
+    for (int c = threadIdx.x; c < nc; c += blockDim.x) { s_w[c] = pm[base + c]; s_l[c] = pl[base + c]; }
+    __syncthreads();
     float M = -CUDART_INF_F;
-    for (int c = 0; c < nc; ++c) M = fmaxf(M, pm[base + c]);
-    float L = 0.0f, o = 0.0f;
-    for (int c = 0; c < nc; ++c) {
-        const float w = exp2f(pm[base + c] - M);            // partial maxima are in the base-2 domain
-        L = fmaf(pl[base + c], w, L);
-        o = fmaf(po[(base + c) * hd + dim], w, o);
+    for (int c = 0; c < nc; ++c) M = fmaxf(M, s_w[c]);
+    __syncthreads();
+    for (int c = threadIdx.x; c < nc; c += blockDim.x) s_w[c] = exp2f(s_w[c] - M);     // partial maxima are in the base-2 domain
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float L = 0.0f;
+        for (int c = 0; c < nc; ++c) L = fmaf(s_l[c], s_w[c], L);
+        s_L = L;
     }
-    bf16 hi, lo;
-    split_bf16(o / L, hi, lo);
-    const size_t out = (size_t)row * Hq * hd + head * hd + dim;
-    ao_hi[out] = hi;
-    ao_lo[out] = lo;
+    float o = 0.0f;
+    for (int c0 = slice; c0 < nc; c0 += 4 * COMBINE_SLICES) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = c0 + u * COMBINE_SLICES;
+            v[u] = (c < nc) ? po[(base + c) * hd + dim] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = c0 + u * COMBINE_SLICES;
+            if (c < nc) o = fmaf(v[u], s_w[c], o);
+        }
+    }
+    s_o[slice][dim] = o;
+    __syncthreads();
+    if (slice == 0) {
+        float t = s_o[0][dim];
+        for (int k = 1; k < COMBINE_SLICES; ++k) t += s_o[k][dim];
+        bf16 hi, lo;
+        split_bf16(t / s_L, hi, lo);
+        const size_t out = (size_t)row * Hq * hd + head * hd + dim;
+        ao_hi[out] = hi;
+        ao_lo[out] = lo;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -695,7 +729,7 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
                                                                             ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, ws.attn_m,
                                                                             ws.attn_l, ws.attn_o)));
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
+           (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
     return ANPD_OK;
 }
