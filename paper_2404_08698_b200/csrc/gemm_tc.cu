@@ -180,17 +180,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tma_load_2d(sa, &map_w, 0, (int)((i * gridDim.x + blockIdx.x) * TILE_M), &bar_full[i], pol_w);
             }
             pdl_wait();
+            int kb = (int)(lo % g.k_blocks);            // k-block of the next activation load; advanced without divisions
             for (long long i = 0; i < ahead; ++i) {
                 unsigned char* sa = smem + (size_t)i * stage_bytes;
-                const int kb = (int)((lo + i) % g.k_blocks);
                 tma_load_2d(sa + A_BYTES, &map_hi, kb * TILE_K, 0, &bar_full[i], pol_a);
                 tma_load_2d(sa + A_BYTES + g.NB * 128, &map_lo, kb * TILE_K, 0, &bar_full[i], pol_a);
+                if (++kb == g.k_blocks) kb = 0;
             }
             issued = ahead;
             stage = (int)(ahead % g.stages);
             phase = (ahead == g.stages) ? 1u : 0u;
             for (long long blk = lo + ahead; blk < hi && ok; ++blk) {
-                const int kb = (int)(blk % g.k_blocks);
                 ok = mbar_wait(&bar_empty[stage], phase ^ 1u, abortp);
                 if (!ok) break;
                 unsigned char* sa = smem + (size_t)stage * stage_bytes;
@@ -198,6 +198,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tma_load_2d(sa, &map_w, 0, (int)(((blk - lo) * gridDim.x + blockIdx.x) * TILE_M), &bar_full[stage], pol_w);   // this CTA's slot of the step's window
                 tma_load_2d(sa + A_BYTES, &map_hi, kb * TILE_K, 0, &bar_full[stage], pol_a);
                 tma_load_2d(sa + A_BYTES + g.NB * 128, &map_lo, kb * TILE_K, 0, &bar_full[stage], pol_a);
+                if (++kb == g.k_blocks) kb = 0;
                 ++issued;
                 if (++stage == g.stages) { stage = 0; phase ^= 1u; }
             }
