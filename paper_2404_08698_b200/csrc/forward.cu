@@ -722,12 +722,15 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
         CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_set = true;
     }
-    dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
-    LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_partial_kernel<HD>, grid, ATTN_THREADS, smem, m->stream, ws.q_hi, ws.q_lo, kv->kpool + layer * layer_elems,
-                                                                            kv->vpool + layer * layer_elems, kv->page_table, kv->pages_per_seq,
-                                                                            ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, ws.attn_m,
-                                                                            ws.attn_l, ws.attn_o)));
+    if (HD == 128 && kv->attn_tc) {
+        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos));
+    } else {
+        dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
+        LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
+               (launch_k(attn_partial_kernel<HD>, grid, ATTN_THREADS, smem, m->stream, ws.q_hi, ws.q_lo, kv->kpool + layer * layer_elems,
+                         kv->vpool + layer * layer_elems, kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads,
+                         c.n_kv_heads, ws.attn_m, ws.attn_l, ws.attn_o)));
+    }
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));

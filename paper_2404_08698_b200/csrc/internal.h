@@ -226,6 +226,8 @@ struct anpd_kv {
     anpd_model* m;
     int batch, max_len, pages_per_seq, total_pages;
     __nv_bfloat16 *kpool, *vpool;     // per layer and page: K [Hkv][KV_PAGE][hd]; V transposed [Hkv][hd][KV_PAGE]
+    CUtensorMap map_k, map_v;         // TMA views of the two pools as [all page rows][hd] matrices (head dimension 128 only)
+    bool attn_tc;                     // attention on tcgen05 (head dimension 128); otherwise the mma.sync kernel
     int* page_table;                  // device [batch][pages_per_seq]
     float *rope_cos, *rope_sin;       // [max_len][hd/2]
     SeqState* seq;                    // device [batch]
@@ -258,6 +260,9 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
 // `seq` gives the first generated token, kv_len becomes prompt_len.  d_ctxs may be null; otherwise
 // accepted tokens and the next token are appended to the sequences' token buffers.
 anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len);
+
+// attn_tc.cu: per-page attention partials for head dimension 128 (same outputs as the mma.sync kernel in forward.cu)
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos);
 
 // gemm_tc.cu
 anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, int box_rows, bool streamed);

@@ -150,6 +150,9 @@ def test_page_order_does_not_matter(A):
     (ModelShape(2, 128, 8, 2, 64, 200, 512), 150),      # grouped-query, 4 q heads per kv head, hd 64
     (ModelShape(1, 256, 2, 2, 128, 264, 300), 131),     # hd 128, ragged vocab / ffn
     (ModelShape(2, 128, 8, 1, 64, 136, 1030), 9),       # 8 q heads on one kv head, prompt shorter than a pass
+    (ModelShape(2, 256, 4, 2, 128, 264, 300), 200),     # hd 128 (tensor-memory attention), 2 q heads per kv head, two key pages
+    (ModelShape(1, 256, 4, 1, 128, 136, 300), 140),     # hd 128, 4 q heads on one kv head
+    (ModelShape(1, 256, 8, 1, 128, 136, 300), 130),     # hd 128, 8 q heads on one kv head
 ])
 def test_other_shapes_logits_parity(A, shape, plen):
     r = Rig(A, shape, seed=11, std=0.05, jitter=0.1, max_len=256)
