@@ -1,7 +1,7 @@
 // Attention of the verify step for head dimension 128 on the sm_100a tensor cores
 // (paper Section 3.1, "Verification": the K+1 rows of a step attend to the cached keys).
 //
-// One CTA handles one 128-key page of one kv head for one group of 8 rows.  With so few query rows
+// A work item is one 128-key page of one kv head for one group of 8 rows.  With so few query rows
 // the operands are swapped, as in the weight GEMM: the page is the MMA's 128-row M operand and the
 // 8 x G query vectors that share the kv head are its N operand.
 //   S^T [128 keys x N]  = K page   [128 keys x 128 dims] . Q^T     (tcgen05.mma, accumulator in tensor memory)
@@ -10,17 +10,27 @@
 // TMA in the 128-byte-swizzled layout the MMA reads.  Queries and softmax weights enter as two bf16
 // terms each (hi rows then lo rows of the N operand, N = 2 x 8 x G), so only the cache's own bf16
 // rounding is left; the two halves of an accumulator are added when it is read back.
-// Thread t of the CTA owns tensor-memory lane t: key t of the page after the first product, output
+//
+// The kernel is persistent: one CTA per SM holds up to five independent "slots" (a warpgroup of
+// 128 threads with its own 32 KB page buffer, operand staging and tensor-memory columns), and a
+// slot walks through its share of the items.  The page buffer first receives the K page; as soon as
+// the first product has consumed it the V^T page is requested into the same buffer and lands while
+// the softmax runs; after the second product the next item's K page follows.  With five slots per
+// SM every SM keeps several page copies in flight, and at the context lengths of interest each slot
+// has one or two items.
+// Thread t of a slot owns tensor-memory lane t: key t of the page after the first product, output
 // dimension t after the second.  The softmax over the page's keys is a reduction across threads
 // (shuffle tree inside a warp, then the four warps in warp order).  Each page leaves a partial
 // (max, sum, weighted values) per query vector; the combine kernel merges pages in page order.
 // Every value depends on the row's own position and inputs only: masked keys contribute exact zeros
 // and the order of every sum is fixed by key positions, so a row's result does not depend on which
-// other rows share the launch.
+// other rows share the launch, nor on which slot handled the page.
 #include "internal.h"
 #include "tc_ptx.cuh"
 
 #include <math_constants.h>
+
+#include <algorithm>
 
 typedef __nv_bfloat16 bf16;
 
@@ -30,7 +40,6 @@ using namespace tc;
 
 constexpr int HD = 128;
 constexpr int PAGE_ATOM = 128 * 128;        // bytes of a 128-row x 64-column bf16 tile (one TMA box)
-constexpr int ATTN_TC_THREADS = 128;
 constexpr int ATTN_ERR_TIMEOUT = 202;
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -43,93 +52,156 @@ __device__ __forceinline__ int b_operand_offset(int n, int k) {
     return (k >> 6) * (N * 128) + (n >> 3) * 1024 + (n & 7) * 128 + ((((kk >> 3) ^ (n & 7))) << 4) + (kk & 7) * 2;
 }
 
+// Slots per CTA for G query heads per kv head: what fits in shared memory and tensor memory.
+template <int G> struct AttnCfg {
+    static constexpr int Q = 8 * G;                      // query vectors: 8 rows x G heads of the group
+    static constexpr int N = 2 * Q;                      // MMA N: hi terms then lo terms
+    static constexpr int B_BYTES = N * 256;              // one N-row operand (two 64-column tiles)
+    static constexpr int SLOT_BYTES = 2 * PAGE_ATOM + 2 * B_BYTES;       // page buffer (K, then V), Q operand, P operand
+    static constexpr int SLOTS = (G == 1) ? 5 : (G == 2) ? 4 : (G == 4) ? 3 : 2;
+    static constexpr int THREADS = SLOTS * 128;
+    static constexpr int TMEM_NEED = SLOTS * N;          // per slot N columns: S^T, then O^T in the same columns
+    static constexpr int TMEM_COLS = TMEM_NEED <= 32 ? 32 : TMEM_NEED <= 64 ? 64 : TMEM_NEED <= 128 ? 128 : TMEM_NEED <= 256 ? 256 : 512;
+    static constexpr size_t SMEM = (size_t)SLOTS * SLOT_BYTES + 1024;
+};
+
+__device__ __forceinline__ void slot_bar(int slot) { asm volatile("bar.sync %0, 128;" ::"r"(slot + 1) : "memory"); }
+
+struct AttnItem { int c, kvh, r0, pos_lo, seq; };
+
 template <int G>
-__global__ void __launch_bounds__(ATTN_TC_THREADS)
+__global__ void __launch_bounds__(AttnCfg<G>::THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const bf16* __restrict__ q_hi,
                const bf16* __restrict__ q_lo, const int* __restrict__ page_table, int pages_per_seq, const int* __restrict__ row_pos,
-               const int* __restrict__ row_seq, int Hq, int Hkv, int layer_row0, float* __restrict__ pm, float* __restrict__ pl,
-               float* __restrict__ po, int* err) {
-    constexpr int Q = 8 * G;                 // query vectors: 8 rows x G heads of the group
-    constexpr int N = 2 * Q;                 // MMA N: hi terms then lo terms
-    constexpr int B_BYTES = N * 256;         // one N-row operand (two 64-column tiles)
-    constexpr int TMEM_COLS = (2 * N < 32) ? 32 : 2 * N;      // S^T in columns [0, N), O^T in [N, 2N)
+               const int* __restrict__ row_seq, int Hq, int Hkv, int layer_row0, int chunks, int n_items, float* __restrict__ pm,
+               float* __restrict__ pl, float* __restrict__ po, int* err) {
+    typedef AttnCfg<G> Cfg;
+    constexpr int Q = Cfg::Q, N = Cfg::N, SLOTS = Cfg::SLOTS;
     extern __shared__ __align__(1024) unsigned char attn_tc_smem[];
-    __shared__ uint64_t bar_kv, bar_s, bar_o;
+    __shared__ uint64_t bar_k[SLOTS], bar_v[SLOTS], bar_s[SLOTS], bar_o[SLOTS];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float red[4][Q];
+    __shared__ float red_max[SLOTS][4][Q];
+    __shared__ float red_sum[SLOTS][2][4][Q];
 
     pdl_trigger();
-    unsigned char* smem = attn_tc_smem + ((1024u - (smem_u32(attn_tc_smem) & 1023u)) & 1023u);
-    unsigned char* Ks = smem;                        // two tiles: dims 0..63, dims 64..127
-    unsigned char* Vs = smem + 2 * PAGE_ATOM;        // two tiles: keys 0..63, keys 64..127
-    unsigned char* Qs = smem + 4 * PAGE_ATOM;
-    unsigned char* Ps = Qs + B_BYTES;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int c = blockIdx.x, kvh = blockIdx.y, r0 = blockIdx.z * ANPD_ROWS;
+    const int slot = threadIdx.x >> 7, t = threadIdx.x & 127, warp = t >> 5, lane = t & 31;
+    unsigned char* smem = attn_tc_smem + ((1024u - (smem_u32(attn_tc_smem) & 1023u)) & 1023u) + (size_t)slot * Cfg::SLOT_BYTES;
+    unsigned char* Bs = smem;                        // the K page (tiles: dims 0..63, 64..127), later the V^T page (keys 0..63, 64..127)
+    unsigned char* Qs = smem + 2 * PAGE_ATOM;
+    unsigned char* Ps = Qs + Cfg::B_BYTES;
 
-    if (tid == 0) {
+    if (threadIdx.x == 0) {
         abort_flag = 0;
-        mbar_init(&bar_kv, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
+        for (int i = 0; i < SLOTS; ++i) { mbar_init(&bar_k[i], 1); mbar_init(&bar_v[i], 1); mbar_init(&bar_s[i], 1); mbar_init(&bar_o[i], 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *((volatile uint32_t*)&tmem_slot);
+    const uint32_t tmem_base = *((volatile uint32_t*)&tmem_slot) + (uint32_t)(slot * N);
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
     volatile int* abortp = &abort_flag;
-
-    pdl_wait();                                      // the row plan, the queries and this step's K/V rows come from earlier kernels
-    const int pos_lo = row_pos[r0], pos_hi = row_pos[r0 + ANPD_ROWS - 1];
-    const bool active = c * KV_PAGE <= pos_hi;       // block-uniform: pages beyond the last row's position hold nothing any row may see
-    bool ok = true;
     // fp32 accumulate, bf16 x bf16, both operands K-major, M = 128
     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-    if (active) {
-        if (tid == 0) {
-            const int page = page_table[row_seq[r0] * pages_per_seq + c];
-            const int row = layer_row0 + (page * Hkv + kvh) * KV_PAGE;       // first row of the page in the pools' 2-D view
-            const uint64_t pol = policy_evict_first();
-            mbar_expect_tx(&bar_kv, 4 * PAGE_ATOM);
-            tma_load_2d(Ks, &map_k, 0, row, &bar_kv, pol);
-            tma_load_2d(Ks + PAGE_ATOM, &map_k, 64, row, &bar_kv, pol);
-            tma_load_2d(Vs, &map_v, 0, row, &bar_kv, pol);
-            tma_load_2d(Vs + PAGE_ATOM, &map_v, 64, row, &bar_kv, pol);
-        }
-        // queries: row n of the operand is query vector n % Q (hi term for n < Q, lo term after); 16-byte chunks
-        for (int idx = tid; idx < N * 16; idx += ATTN_TC_THREADS) {
-            const int n = idx >> 4, c16 = idx & 15;
-            const int qn = n % Q, g = qn >> 3, r = qn & 7;
-            const bf16* src = (n < Q ? q_hi : q_lo) + (size_t)(r0 + r) * Hq * HD + (size_t)(kvh * G + g) * HD + c16 * 8;
-            *(uint4*)(Qs + b_operand_offset<N>(n, c16 * 8)) = *(const uint4*)src;
-        }
-        fence_async_smem();
-        __syncthreads();
+    const uint64_t pol = policy_evict_first();
 
-        if (tid == 0) {
-            ok = mbar_wait(&bar_kv, 0, abortp);
-            if (ok) {
+    pdl_wait();                                      // the row plan, the queries and this step's K/V rows come from earlier kernels
+
+    // Item `it` -> (page, kv head, row group); pages beyond the group's last position hold nothing a row may see.
+    const int stride = gridDim.x * SLOTS;
+    auto decode = [&](int it, AttnItem& out) {
+        const int rest = it / chunks;
+        out.c = it % chunks; out.kvh = rest % Hkv; out.r0 = (rest / Hkv) * ANPD_ROWS;
+    };
+    auto next_item = [&](int it, AttnItem& out) -> int {
+        for (; it < n_items; it += stride) {
+            decode(it, out);
+            const int hi = row_pos[out.r0 + ANPD_ROWS - 1];          // three independent loads
+            out.pos_lo = row_pos[out.r0];
+            out.seq = row_seq[out.r0];
+            if (out.c * KV_PAGE <= hi) return it;
+        }
+        return n_items;
+    };
+    auto page_row = [&](const AttnItem& a) -> int {   // first row of the item's page in the pools' 2-D view
+        return layer_row0 + (page_table[a.seq * pages_per_seq + a.c] * Hkv + a.kvh) * KV_PAGE;
+    };
+    auto load_page = [&](const CUtensorMap* map, uint64_t* bar, const AttnItem& a) {
+        const int row = page_row(a);
+        mbar_expect_tx(bar, 2 * PAGE_ATOM);
+        tma_load_2d(Bs, map, 0, row, bar, pol);
+        tma_load_2d(Bs + PAGE_ATOM, map, 64, row, bar, pol);
+    };
+    // queries: row n of the operand is query vector n % Q (hi term for n < Q, lo term after); 16-byte chunks
+    constexpr int QCH = (N * 16 + 127) / 128;
+    auto fetch_q = [&](const AttnItem& a, uint4* regs) {
+#pragma unroll
+        for (int u = 0; u < QCH; ++u) {
+            const int idx = t + u * 128;
+            if (idx < N * 16) {
+                const int n = idx >> 4, c16 = idx & 15;
+                const int qn = n % Q, g = qn >> 3, r = qn & 7;
+                const bf16* src = (n < Q ? q_hi : q_lo) + (size_t)(a.r0 + r) * Hq * HD + (size_t)(a.kvh * G + g) * HD + c16 * 8;
+                regs[u] = *(const uint4*)src;
+            }
+        }
+    };
+    auto stage_q = [&](const uint4* regs) {
+#pragma unroll
+        for (int u = 0; u < QCH; ++u) {
+            const int idx = t + u * 128;
+            if (idx < N * 16) *(uint4*)(Qs + b_operand_offset<N>(idx >> 4, (idx & 15) * 8)) = regs[u];
+        }
+    };
+
+    AttnItem cur, nxt;
+    int it = blockIdx.x * SLOTS + slot;
+    uint32_t k_issued = 0, v_issued = 0;             // page loads requested by this slot's first thread
+    if (it < n_items) {
+        // the queries of the slot's first candidate are requested before anything that has to wait for the row plan
+        uint4 qr[QCH];
+        decode(it, cur);
+        fetch_q(cur, qr);
+        const int first = it;
+        it = next_item(it, cur);
+        if (it < n_items) {
+            if (t == 0) { load_page(&map_k, &bar_k[slot], cur); k_issued = 1; }
+            if (it != first) fetch_q(cur, qr);
+            stage_q(qr);
+            fence_async_smem();
+            slot_bar(slot);
+        }
+    }
+    for (uint32_t j = 0; it < n_items; ++j) {
+        const uint32_t par = j & 1u;
+        const int it_next = next_item(it + stride, nxt);
+        const bool more = it_next < n_items;
+        // ---- S^T = K . Q^T ----
+        if (t == 0) {
+            if (mbar_wait(&bar_k[slot], par, abortp)) {
                 tc_fence_after();
 #pragma unroll
                 for (int k16 = 0; k16 < HD / 16; ++k16) {
                     const uint64_t adv = (uint64_t)((k16 & 3) * 2);                 // 32 bytes along K inside the swizzle row, 16-byte units
-                    tc_mma_bf16(tmem_base, make_smem_desc(smem_u32(Ks + (k16 >> 2) * PAGE_ATOM)) + adv,
+                    tc_mma_bf16(tmem_base, make_smem_desc(smem_u32(Bs + (k16 >> 2) * PAGE_ATOM)) + adv,
                                 make_smem_desc(smem_u32(Qs + (k16 >> 2) * (N * 128))) + adv, idesc, k16 > 0 ? 1u : 0u);
                 }
-                tc_commit(&bar_s);
+                tc_commit(&bar_s[slot]);
             }
         }
-        ok = mbar_wait(&bar_s, 0, abortp) && ok;
-        ok = __syncthreads_and(ok) != 0;
-    }
-    if (active && ok) {
+        mbar_wait(&bar_s[slot], par, abortp);
         tc_fence_after();
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // the first product is done with the page buffer and the query staging: the V^T page takes the buffer,
+        // and the next item's queries are requested
+        if (t == 0) { load_page(&map_v, &bar_v[slot], cur); ++v_issued; }
+        uint4 qr[QCH];
+        if (more) fetch_q(nxt, qr);
         float s[Q];
         {
             float v[N];
@@ -138,95 +210,105 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
 #pragma unroll
             for (int q = 0; q < Q; ++q) s[q] = v[q] + v[Q + q];
         }
-        // mask by position (this thread's key is c * 128 + tid), maximum over the page's keys per query vector
-        const int key = c * KV_PAGE + tid;
+        // mask by position (this thread's key is c * 128 + t), maximum over the page's keys per query vector
+        const int key = cur.c * KV_PAGE + t;
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
-            if (key > pos_lo + (q & 7)) s[q] = -CUDART_INF_F;
+            if (key > cur.pos_lo + (q & 7)) s[q] = -CUDART_INF_F;
             float mx = s[q];
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            if (lane == 0) red[warp][q] = mx;
+            if (lane == 0) red_max[slot][warp][q] = mx;
         }
-        __syncthreads();
+        tc_fence_before();
+        slot_bar(slot);
+        // weights (base-2 domain: the queries carry log2(e) / sqrt(hd)), their sum, and the P operand
         float m[Q];
 #pragma unroll
-        for (int q = 0; q < Q; ++q) m[q] = fmaxf(fmaxf(red[0][q], red[1][q]), fmaxf(red[2][q], red[3][q]));
-        __syncthreads();
-        // weights (base-2 domain: the queries carry log2(e) / sqrt(hd)), their sum, and the P operand
-#pragma unroll
         for (int q = 0; q < Q; ++q) {
+            m[q] = fmaxf(fmaxf(red_max[slot][0][q], red_max[slot][1][q]), fmaxf(red_max[slot][2][q], red_max[slot][3][q]));
             const float p = (m[q] == -CUDART_INF_F) ? 0.0f : exp2f(s[q] - m[q]);
             const bf16 h = __float2bfloat16_rn(p);
             const bf16 l = __float2bfloat16_rn(p - __bfloat162float(h));
-            *(bf16*)(Ps + b_operand_offset<N>(q, tid)) = h;
-            *(bf16*)(Ps + b_operand_offset<N>(Q + q, tid)) = l;
+            *(bf16*)(Ps + b_operand_offset<N>(q, t)) = h;
+            *(bf16*)(Ps + b_operand_offset<N>(Q + q, t)) = l;
             float sum = p;
             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) red[warp][q] = sum;
+            if (lane == 0) red_sum[slot][par][warp][q] = sum;
         }
+        if (more) stage_q(qr);
         fence_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
+        slot_bar(slot);
+        // ---- O^T = V^T . P^T (into the columns S^T occupied: every thread has read its scores) ----
+        if (t == 0) {
+            if (mbar_wait(&bar_v[slot], par, abortp)) {
+                tc_fence_after();
 #pragma unroll
-            for (int k16 = 0; k16 < KV_PAGE / 16; ++k16) {
-                const uint64_t adv = (uint64_t)((k16 & 3) * 2);
-                tc_mma_bf16(tmem_base + (uint32_t)N, make_smem_desc(smem_u32(Vs + (k16 >> 2) * PAGE_ATOM)) + adv,
-                            make_smem_desc(smem_u32(Ps + (k16 >> 2) * (N * 128))) + adv, idesc, k16 > 0 ? 1u : 0u);
+                for (int k16 = 0; k16 < KV_PAGE / 16; ++k16) {
+                    const uint64_t adv = (uint64_t)((k16 & 3) * 2);
+                    tc_mma_bf16(tmem_base, make_smem_desc(smem_u32(Bs + (k16 >> 2) * PAGE_ATOM)) + adv,
+                                make_smem_desc(smem_u32(Ps + (k16 >> 2) * (N * 128))) + adv, idesc, k16 > 0 ? 1u : 0u);
+                }
+                tc_commit(&bar_o[slot]);
             }
-            tc_commit(&bar_o);
         }
-        if (tid < Q) {
-            const int q = tid;
-            const size_t out = ((size_t)(r0 + (q & 7)) * Hq + (kvh * G + (q >> 3))) * pages_per_seq + c;
-            pm[out] = m[q];
-            pl[out] = (red[0][q] + red[1][q]) + (red[2][q] + red[3][q]);
+        if (t < Q) {
+            const size_t out = ((size_t)(cur.r0 + (t & 7)) * Hq + (cur.kvh * G + (t >> 3))) * pages_per_seq + cur.c;
+            float mt = m[0];
+#pragma unroll
+            for (int q = 1; q < Q; ++q) mt = (q == t) ? m[q] : mt;
+            pm[out] = mt;
+            pl[out] = (red_sum[slot][par][0][t] + red_sum[slot][par][1][t]) + (red_sum[slot][par][2][t] + red_sum[slot][par][3][t]);
         }
-        ok = mbar_wait(&bar_o, 0, abortp);
-        if (ok) {
-            tc_fence_after();
+        mbar_wait(&bar_o[slot], par, abortp);
+        tc_fence_after();
+        if (more && t == 0) { load_page(&map_k, &bar_k[slot], nxt); ++k_issued; }        // the second product is done with the page buffer
+        {
             float v[N];
 #pragma unroll
-            for (int c0 = 0; c0 < N; c0 += 16) tc_ld16(lane_base + (uint32_t)(N + c0), v + c0);
+            for (int c0 = 0; c0 < N; c0 += 16) tc_ld16(lane_base + (uint32_t)c0, v + c0);
 #pragma unroll
             for (int q = 0; q < Q; ++q) {
-                const size_t out = ((size_t)(r0 + (q & 7)) * Hq + (kvh * G + (q >> 3))) * pages_per_seq + c;
-                po[out * HD + tid] = v[q] + v[Q + q];
+                const size_t out = ((size_t)(cur.r0 + (q & 7)) * Hq + (cur.kvh * G + (q >> 3))) * pages_per_seq + cur.c;
+                po[out * HD + t] = v[q] + v[Q + q];
             }
         }
+        tc_fence_before();
+        if (more) slot_bar(slot);                    // the next first product overwrites the columns just read
+        cur = nxt;
+        it = it_next;
     }
-    if (active && tid == 0 && abort_flag) {
-        // gave up somewhere: let the page copies land before the CTA may exit
-        for (unsigned spin = 0; spin < WAIT_LIMIT && !mbar_try_wait(&bar_kv, 0); ++spin) {}
-        atomicExch(err, ATTN_ERR_TIMEOUT);
+    if (t == 0 && abort_flag) {
+        // gave up somewhere: let the last page copies land before the CTA may exit
+        if (k_issued) for (unsigned spin = 0; spin < WAIT_LIMIT && !mbar_try_wait(&bar_k[slot], (k_issued - 1) & 1u); ++spin) {}
+        if (v_issued) for (unsigned spin = 0; spin < WAIT_LIMIT && !mbar_try_wait(&bar_v[slot], (v_issued - 1) & 1u); ++spin) {}
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (threadIdx.x == 0 && abort_flag) atomicExch(err, ATTN_ERR_TIMEOUT);
+    if (threadIdx.x < 32) {
         tc_fence_after();
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*((volatile uint32_t*)&tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
     }
 }
 
 template <int G>
 anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int chunks) {
+    typedef AttnCfg<G> Cfg;
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
-    constexpr int N = 16 * G;
-    const size_t smem = 4 * PAGE_ATOM + 2 * (size_t)N * 256 + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
         attr_set = true;
     }
     const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
-    dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
+    const int n_items = chunks * c.n_kv_heads * (rows / ANPD_ROWS);
+    const int grid = std::min(m->num_sms, (n_items + Cfg::SLOTS - 1) / Cfg::SLOTS);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_tc_kernel<G>, grid, ATTN_TC_THREADS, smem, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
-                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, ws.attn_m, ws.attn_l, ws.attn_o,
-                     ws.gemm_err)));
+           (launch_k(attn_tc_kernel<G>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
+                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
+                     ws.attn_l, ws.attn_o, ws.gemm_err)));
     return ANPD_OK;
 }
 
