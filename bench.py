@@ -201,6 +201,70 @@ def verify_microbench(args, A, wl, model, stream) -> None:
                       "rows": rows_out}))
 
 
+def batch_generate_bench(args, A, wl, model, stream, t_setup0: float) -> None:
+    """Workloads with several independent sequences (C5): every verify step carries 8 rows per sequence,
+    each sequence has its own n-gram tables, KV pages, draft and acceptance; one weight stream serves
+    all of them.  Timed through the host-buffer call (the only batched entry point), with CUDA events
+    on the library's stream; the host<->device copies of prompts and outputs are inside."""
+    shape, B = wl.shape, wl.batch
+    max_len = wl.prompt_len + wl.max_new + 64
+    kv = A.anpd_kv_create(model, max_len, B)
+    ctxs = [A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, stream.cuda_stream) for _ in range(B)]
+    prompts = np.stack(make_prompts(wl))
+    torch.cuda.synchronize()
+    t_setup = time.perf_counter() - t_setup0
+
+    def timed(K: int, steps: int, warmup: int):
+        out = st = None
+        for _ in range(warmup):
+            out, st = A.anpd_generate_batch(model, kv, ctxs, prompts, wl.max_new, K)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        e0.record(stream)
+        for _ in range(steps):
+            out, st = A.anpd_generate_batch(model, kv, ctxs, prompts, wl.max_new, K)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 1e3, time.perf_counter() - t0, out, st
+
+    timed(wl.K, 0, max(args.warmup, 1))
+    sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    A.anpd_launch_count(True)
+    sampler.start()
+    t_anpd, wall_anpd, out_anpd, st_anpd = timed(wl.K, args.steps, 0)
+    clocks = sampler.stop()
+    launches = A.anpd_launch_count(True)
+    t_greedy, _, out_greedy, st_greedy = timed(0, args.steps, 1)
+    tokens = args.steps * B * wl.max_new
+    acc = sum(s["accepted"] for s in st_anpd)
+    steps_sum = sum(s["steps"] for s in st_anpd)
+    drafted = sum(s["drafted"] for s in st_anpd)
+    result = {
+        "metric": f"tokens_per_s_bs{B}_anpd", "value": tokens / t_anpd, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t_anpd / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name}: {shape.n_layers}L d{shape.d_model} {shape.n_q_heads}q/{shape.n_kv_heads}kv x{shape.head_dim} "
+                               f"ffn{shape.d_ffn} vocab{shape.vocab}, {B} sequences, prompt {wl.prompt_len}, {wl.max_new} new tokens each",
+                   "n_max": wl.n_max, "K": wl.K, "parallelism": "single GPU", "l2": "inputs (weights) far larger than L2; no flush",
+                   "step": f"one anpd_generate_batch run ({B} prefills + the shared decode loop)"},
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+        "e2e": {"value": tokens / wall_anpd, "unit": UNIT, "h2d_bytes_per_step": int(prompts.nbytes), "d2h_bytes_per_step": int(out_anpd.nbytes)},
+        "gpu_launches": int(launches),
+        "anpd": {"tokens_per_s": tokens / t_anpd, "decode_steps_per_sequence": [s["steps"] for s in st_anpd],
+                 "mean_accepted_per_step": acc / max(steps_sum, 1), "hit_ratio_alpha": acc / max(drafted, 1),
+                 "ms_prefill": st_anpd[0]["ms_prefill"], "ms_decode": st_anpd[0]["ms_decode"]},
+        "greedy": {"tokens_per_s": tokens / t_greedy, "ms_prefill": st_greedy[0]["ms_prefill"], "ms_decode": st_greedy[0]["ms_decode"]},
+        "speedup_vs_greedy": t_greedy / t_anpd,
+        "anpd_equals_greedy": bool(np.array_equal(out_anpd, out_greedy)),
+        "setup_s": t_setup,
+    }
+    print(json.dumps(result))
+    for c in ctxs:
+        A.anpd_ngram_destroy(c)
+    A.anpd_kv_destroy(kv)
+
+
 def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
     """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
     time.  `dist` is torch.distributed (or None for one process)."""
@@ -259,6 +323,12 @@ def main() -> None:
     torch.cuda.empty_cache()
     if args.mode == "verify":
         verify_microbench(args, A, wl, model, stream)
+        A.anpd_model_destroy(model)
+        return
+    if wl.batch > 1:
+        if world > 1:
+            raise SystemExit("the batched workload is a single-GPU line")
+        batch_generate_bench(args, A, wl, model, stream, t_setup)
         A.anpd_model_destroy(model)
         return
     max_len = wl.prompt_len + wl.max_new + 64

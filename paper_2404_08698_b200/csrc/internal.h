@@ -155,7 +155,7 @@ anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batc
 // model, KV cache and workspace
 // ---------------------------------------------------------------------------------------------
 constexpr int KV_PAGE = 128;          // positions per KV page (= key chunk of one attention block)
-constexpr int PREFILL_ROWS = 64;      // rows per prefill pass
+constexpr int PREFILL_ROWS = 128;     // rows per prefill pass (the MMA takes hi and lo rows side by side: N = 256, its maximum)
 
 // How one [N][K] weight matrix is cut across the persistent GEMM CTAs (depends on the shape and the
 // SM count only): tile t is started by CTA first_cta[t] and covered by seg_count[t] consecutive CTAs,
