@@ -161,7 +161,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     };
 
     AttnItem cur, nxt;
-    int it = blockIdx.x * SLOTS + slot;
+    int it = slot * gridDim.x + blockIdx.x;          // consecutive items go to different SMs: every SM gets its share of slots in use
     uint32_t k_issued = 0, v_issued = 0;             // page loads requested by this slot's first thread
     if (it < n_items) {
         // the queries of the slot's first candidate are requested before anything that has to wait for the row plan
@@ -304,7 +304,7 @@ anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int 
     }
     const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
     const int n_items = chunks * c.n_kv_heads * (rows / ANPD_ROWS);
-    const int grid = std::min(m->num_sms, (n_items + Cfg::SLOTS - 1) / Cfg::SLOTS);
+    const int grid = std::min(m->num_sms, n_items);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (launch_k(attn_tc_kernel<G>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
                      kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
