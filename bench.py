@@ -265,6 +265,10 @@ def batch_generate_bench(args, A, wl, model, stream, t_setup0: float) -> None:
     A.anpd_kv_destroy(kv)
 
 
+# Mean DRAM bytes (read + write) per weight-GEMM launch of one verify step, from the ncu capture summarised in
+# profiles/gemm_tc_kernel_7B_2layer_ncu.md (one layer's four projections and the LM head, scaled to 32 layers).
+NCU_GEMM_TRAFFIC_PER_LAUNCH = {"C3": 105.1e6}
+
 def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
     """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
     time.  `dist` is torch.distributed (or None for one process)."""
@@ -424,7 +428,7 @@ def main() -> None:
     gemm_gbs = prof["gemm_bytes"] / (prof["ms_gemm"] * 1e-3) / 1e9 if prof["ms_gemm"] > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections + LM head)",
                 "achieved": gemm_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                "frac": gemm_gbs / peak, "traffic": None,
+                "frac": gemm_gbs / peak, "traffic": NCU_GEMM_TRAFFIC_PER_LAUNCH.get(wl.name),
                 "launches": prof["n_gemm"], "avg_launch_us": prof["ms_gemm"] * 1e3 / max(prof["n_gemm"], 1),
                 "bytes_per_launch": prof["gemm_bytes"] / max(prof["n_gemm"], 1),
                 "step_share": {"gemm_ms": prof["ms_gemm"] / 5, "attn_ms": prof["ms_attn"] / 5,

@@ -207,3 +207,28 @@ def test_verify_error_paths(A, c1):
     with pytest.raises(A.AnpdError) as e:
         A.anpd_prefill(c1.m, c1.kv, list(range(600)))                  # longer than the cache
     assert e.value.status in (A.ERR_STATE, A.ERR_CAPACITY)
+
+
+def test_tensor_memory_attention_agrees_with_mma_sync_attention(A, monkeypatch):
+    """Head dimension 128 has two attention kernels (tcgen05 with tensor-memory accumulators, and the
+    mma.sync one that head dimension 64 always uses).  They add the keys of a page in different orders,
+    so the logits agree closely but not bit for bit; three key pages, grouped-query heads."""
+    shape = ModelShape(2, 256, 4, 2, 128, 264, 300)
+    prompt = markov_prompt(300, shape.vocab, 2, 9).tolist()
+    w = make_weights(shape, 21, False, std=0.05, norm_gain_jitter=0.1)
+    outs = []
+    for legacy in (False, True):
+        if legacy:
+            monkeypatch.setenv("ANPD_ATTN_MMA_SYNC", "1")
+        else:
+            monkeypatch.delenv("ANPD_ATTN_MMA_SYNC", raising=False)
+        m = gpu_model(A, shape, w)
+        kv = A.anpd_kv_create(m, 512)
+        try:
+            first = A.anpd_prefill(m, kv, prompt)
+            outs.append((first, A.anpd_verify_logits(m, kv, first, prompt[2:9], shape.vocab)))
+        finally:
+            A.anpd_kv_destroy(kv)
+            A.anpd_model_destroy(m)
+    assert outs[0][0] == outs[1][0]
+    assert float(np.abs(outs[0][1] - outs[1][1]).max()) <= 1e-4
