@@ -135,14 +135,6 @@ static anpd_status model_make_plans(anpd_model* m) {
     m->d_ones = m->d_plan_tables + off;
     for (int i = 0; i < max_tiles; ++i) host[off + i] = 1;
     CUDA_TRY(cudaMemcpy(m->d_plan_tables, host.data(), ints * sizeof(int), cudaMemcpyHostToDevice));
-    for (int l = 0; l < c.n_layers; ++l) {
-        LayerW& w = m->layers[l];
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_QKV], w.wqkv, m->plan[GK_QKV]));
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_O], w.wo, m->plan[GK_O]));
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_GU], w.wgu, m->plan[GK_GU]));
-        ANPD_TRY(make_tmap_tiled(&w.map[GK_DOWN], w.wd, m->plan[GK_DOWN]));
-    }
-    ANPD_TRY(make_tmap_tiled(&m->map_lm, m->lm_head, m->plan[GK_LM]));
     return ANPD_OK;
 }
 
@@ -785,11 +777,10 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
         if (plain) {
             ANPD_TRY(gemm_plain_enqueue(plan, dW, dhi, dlo, rows, dpart, N, 0, nullptr));
         } else {
-            CUtensorMap mw, mh, ml;
-            ANPD_TRY(make_tmap_tiled(&mw, dW, plan));
+            CUtensorMap mh, ml;
             ANPD_TRY(make_tmap_bf16(&mh, dhi, rows, K, NB, false));
             ANPD_TRY(make_tmap_bf16(&ml, dlo, rows, K, NB, false));
-            ANPD_TRY(gemm_tc_enqueue(plan, mw, mh, ml, rows, NB, dpart, (size_t)rows * N, N, derr, 0, nullptr));
+            ANPD_TRY(gemm_tc_enqueue(plan, dW, mh, ml, rows, NB, dpart, (size_t)rows * N, N, derr, 0, nullptr));
         }
         CUDA_TRY(cudaDeviceSynchronize());
         int err = 0;

@@ -658,7 +658,7 @@ __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict_
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int k0 = lane * 8; k0 < K; k0 += 256) {
             const long long slot = gemm_block_slot((long long)(n >> 7) * k_blocks + (k0 >> 6), total, G);
-            const uint4 wv = *(const uint4*)(W + ((size_t)slot * 128 + (n & 127)) * 64 + (k0 & 63));
+            const uint4 wv = *(const uint4*)(W + gemm_block_elem(slot, n & 127, k0 & 63));
             const bf16* w8 = (const bf16*)&wv;
             float wf[8];
 #pragma unroll
@@ -702,8 +702,7 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
         *seg_count_out = m->d_ones;
         return gemm_plain_enqueue(plan, W, a_hi, a_lo, rows, ws.part, ws.n_max_out, m->stream, &m->prof);
     }
-    const CUtensorMap& mw = kind == GK_LM ? m->map_lm : m->layers[layer].map[kind];
-    ANPD_TRY(gemm_tc_enqueue(plan, mw, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)ws.r_max * ws.n_max_out,
+    ANPD_TRY(gemm_tc_enqueue(plan, W, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)ws.r_max * ws.n_max_out,
                              ws.n_max_out, ws.gemm_err, m->stream, &m->prof));
     *seg_count_out = plan.d_seg_count;
     return ANPD_OK;

@@ -123,11 +123,10 @@ extern "C" anpd_status anpd_gemm_static(const uint16_t* w_bf16_dev, int N, int K
     static_split_kernel<<<64, 256, 0, st>>>(a_dev, d_hi, d_lo, (size_t)rows * K);
     CUDA_TRY(cudaGetLastError());
     ANPD_TRY(gemm_retile_enqueue(plan, w_bf16_dev, false, N, 0, d_w, st));
-    CUtensorMap mw, mh, ml;
-    ANPD_TRY(make_tmap_tiled(&mw, d_w, plan));
+    CUtensorMap mh, ml;
     ANPD_TRY(make_tmap_bf16(&mh, d_hi, rows, K, NB, false));
     ANPD_TRY(make_tmap_bf16(&ml, d_lo, rows, K, NB, false));
-    ANPD_TRY(gemm_tc_enqueue(plan, mw, mh, ml, rows, NB, d_part, (size_t)rows * N, N, d_err, st, nullptr));
+    ANPD_TRY(gemm_tc_enqueue(plan, d_w, mh, ml, rows, NB, d_part, (size_t)rows * N, N, d_err, st, nullptr));
     static_reduce_kernel<<<64, 256, 0, st>>>(d_part, plan.d_seg_count, rows, N, out_dev);
     CUDA_TRY(cudaGetLastError());
     int err = 0;

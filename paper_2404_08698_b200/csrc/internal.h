@@ -177,7 +177,6 @@ struct LayerW {
     const __nv_bfloat16* wd;          // [d, F]
     const float* attn_norm;           // [d]
     const float* ffn_norm;            // [d]
-    CUtensorMap map[4];               // TMA views of wqkv, wo, wgu, wd (128-row x 64-column boxes)
 };
 
 struct anpd_model {
@@ -191,7 +190,6 @@ struct anpd_model {
     void* slab;
     size_t slab_bytes;
     double streamed_bytes;            // weight bytes one forward reads
-    CUtensorMap map_lm;
     GemmPlan plan[GK_COUNT];
     int* d_plan_tables;               // device copies of the plans' tables
     int* d_ones;                      // [tiles] all 1: segment counts of the plain GEMM
@@ -274,13 +272,18 @@ __host__ __device__ inline long long gemm_block_slot(long long logical, long lon
     const long long c = ((logical + 1) * G + total - 1) / total - 1;      // owner: largest c with c * total / G <= logical
     return (logical - c * total / G) * G + c;
 }
+// Inside its 16 KB slot a block is stored as the shared-memory image the MMA reads: rows of 128 bytes, and
+// within every group of 8 rows the 16-byte chunk c of row r sits at chunk position c ^ (r % 8) (the 128-byte
+// swizzle).  The GEMM brings a block in with one linear copy.  Element (row r, column k) of a block:
+__host__ __device__ inline size_t gemm_block_elem(long long slot, int r, int k) {
+    return ((size_t)slot * 128 + r) * 64 + (size_t)((((k >> 3) ^ (r & 7)) << 3) | (k & 7));
+}
 void gemm_make_plan(GemmPlan* p, int N, int K, int num_sms);
 size_t gemm_tiled_elems(const GemmPlan& p);
-anpd_status make_tmap_tiled(CUtensorMap* out, const void* base_tiled, const GemmPlan& p);
 // Scatters rows [row_off, row_off + rows) of a row-major [rows][K] source (bf16, or fp32 rounded to
 // bf16) into the block storage of the plan's matrix.  The padding must already be zero.
 anpd_status gemm_retile_enqueue(const GemmPlan& p, const void* src, bool src_is_f32, int rows, int row_off, __nv_bfloat16* dst_tiled, cudaStream_t st);
-anpd_status gemm_tc_enqueue(const GemmPlan& plan, const CUtensorMap& map_w, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
+anpd_status gemm_tc_enqueue(const GemmPlan& plan, const __nv_bfloat16* w_blocks, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
                             int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,
                             Profiler* prof);
 // forward.cu: the plain (one warp per output feature) GEMM, kept as a cross-check
