@@ -232,3 +232,41 @@ def test_tensor_memory_attention_agrees_with_mma_sync_attention(A, monkeypatch):
             A.anpd_model_destroy(m)
     assert outs[0][0] == outs[1][0]
     assert float(np.abs(outs[0][1] - outs[1][1]).max()) <= 1e-4
+
+
+def test_long_context_attention_slots_take_several_pages(A, monkeypatch):
+    """93 key pages x 8 kv heads = 744 work items for the persistent tensor-memory attention kernel, more than
+    its 148 x 5 slots on a B200: some slots walk through two pages and reuse their buffers and barriers.  Also
+    the page combine beyond 32 pages.  Checked against the oracle (prompt fed in chunks to bound its memory)
+    and against the mma.sync attention kernel."""
+    shape = ModelShape(1, 256, 8, 8, 128, 264, 300)
+    plen = 92 * 128 + 57
+    prompt = markov_prompt(plen, shape.vocab, 2, 13).tolist()
+    w = make_weights(shape, 23, False, std=0.05, norm_gain_jitter=0.1)
+    draft = prompt[5:12]
+    outs = []
+    for legacy in (False, True):
+        if legacy:
+            monkeypatch.setenv("ANPD_ATTN_MMA_SYNC", "1")
+        else:
+            monkeypatch.delenv("ANPD_ATTN_MMA_SYNC", raising=False)
+        m = gpu_model(A, shape, w)
+        kv = A.anpd_kv_create(m, 96 * 128)
+        try:
+            first = A.anpd_prefill(m, kv, prompt)
+            outs.append((first, A.anpd_verify_logits(m, kv, first, draft, shape.vocab)))
+        finally:
+            A.anpd_kv_destroy(kv)
+            A.anpd_model_destroy(m)
+    assert outs[0][0] == outs[1][0]
+    assert float(np.abs(outs[0][1] - outs[1][1]).max()) <= 1e-4
+    dec = Decoder(shape, as_bf16_values(w), torch.float64)
+    cache = dec.new_cache()
+    lp = None
+    for s in range(0, plen, 1024):
+        lp = dec.forward(prompt[s:s + 1024], cache)
+    if top2_margin(lp[-1]) > MARGIN:
+        assert outs[0][0] == argmax_lowest(lp[-1])
+    want = dec.forward([outs[0][0]] + draft, cache)
+    err = float((torch.from_numpy(outs[0][1]).double() - want).abs().max())
+    assert err <= LOGIT_TOL, err
