@@ -36,7 +36,7 @@ constexpr int TILE_K = 64;              // bf16 elements per k-block = one 128-b
 constexpr int A_BYTES = TILE_M * TILE_K * 2;
 constexpr int GEMM_THREADS = 192;       // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
 constexpr int MAX_STAGES = 12;
-constexpr int RING_STAGES = 6;
+constexpr int RING_STAGES = 5;
 constexpr int GEMM_ERR_TIMEOUT = 201;
 
 struct GemmArgs {
@@ -313,8 +313,8 @@ void gemm_make_plan(GemmPlan* p, int N, int K, int num_sms) {
 
 int gemm_smem_bytes(int NB, int* stages_out) {
     const int stage_bytes = A_BYTES + 2 * NB * 128;
-    // Six 16 KB weight blocks in flight per SM stream fastest on this part (measured: 10 in flight cost 5 % of the
-    // step, 4 cost 2 %); wide activation tiles (prefill) leave room for fewer.
+    // Five 16 KB weight blocks in flight per SM stream fastest on this part (measured: 10 in flight cost 5 % of the
+    // step, 8 cost 3 %, 4 cost 2 %); wide activation tiles (prefill) leave room for fewer.
     int stages = std::min(RING_STAGES, (200 * 1024) / stage_bytes);
     if (stages_out) *stages_out = stages;
     return stages * stage_bytes + 1024;
