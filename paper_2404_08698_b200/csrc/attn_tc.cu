@@ -11,11 +11,11 @@
 // terms each (hi rows then lo rows of the N operand, N = 2 x 8 x G), so only the cache's own bf16
 // rounding is left; the two halves of an accumulator are added when it is read back.
 //
-// The kernel is persistent: one CTA per SM holds up to five independent "slots" (a warpgroup of
+// The kernel is persistent: one CTA per SM holds up to four independent "slots" (a warpgroup of
 // 128 threads with its own 32 KB page buffer, operand staging and tensor-memory columns), and a
 // slot walks through its share of the items.  The page buffer first receives the K page; as soon as
 // the first product has consumed it the V^T page is requested into the same buffer and lands while
-// the softmax runs; after the second product the next item's K page follows.  With five slots per
+// the softmax runs; after the second product the next item's K page follows.  With four slots per
 // SM every SM keeps several page copies in flight, and at the context lengths of interest each slot
 // has one or two items.
 // Thread t of a slot owns tensor-memory lane t: key t of the page after the first product, output
@@ -58,7 +58,7 @@ template <int G> struct AttnCfg {
     static constexpr int N = 2 * Q;                      // MMA N: hi terms then lo terms
     static constexpr int B_BYTES = N * 256;              // one N-row operand (two 64-column tiles)
     static constexpr int SLOT_BYTES = 2 * PAGE_ATOM + 2 * B_BYTES;       // page buffer (K, then V), Q operand, P operand
-    static constexpr int SLOTS = (G == 1) ? 5 : (G == 2) ? 4 : (G == 4) ? 3 : 2;
+    static constexpr int SLOTS = (G <= 2) ? 4 : (G == 4) ? 3 : 2;       // G = 1 would fit five; four measured faster
     static constexpr int THREADS = SLOTS * 128;
     static constexpr int TMEM_NEED = SLOTS * N;          // per slot N columns: S^T, then O^T in the same columns
     static constexpr int TMEM_COLS = TMEM_NEED <= 32 ? 32 : TMEM_NEED <= 64 ? 64 : TMEM_NEED <= 128 ? 128 : TMEM_NEED <= 256 ? 256 : 512;

@@ -236,7 +236,7 @@ def test_tensor_memory_attention_agrees_with_mma_sync_attention(A, monkeypatch):
 
 def test_long_context_attention_slots_take_several_pages(A, monkeypatch):
     """93 key pages x 8 kv heads = 744 work items for the persistent tensor-memory attention kernel, more than
-    its 148 x 5 slots on a B200: some slots walk through two pages and reuse their buffers and barriers.  Also
+    its 148 x 4 slots on a B200: some slots walk through two pages and reuse their buffers and barriers.  Also
     the page combine beyond 32 pages.  Checked against the oracle (prompt fed in chunks to bound its memory)
     and against the mma.sync attention kernel."""
     shape = ModelShape(1, 256, 8, 8, 128, 264, 300)
