@@ -267,7 +267,7 @@ def batch_generate_bench(args, A, wl, model, stream, t_setup0: float) -> None:
 
 # Mean DRAM bytes (read + write) per weight-GEMM launch of one verify step, from the ncu capture summarised in
 # profiles/gemm_tc_kernel_7B_2layer_ncu.md (one layer's four projections and the LM head, scaled to 32 layers).
-NCU_GEMM_TRAFFIC_PER_LAUNCH = {"C3": 105.1e6}
+NCU_GEMM_TRAFFIC_PER_LAUNCH = {"C3": 105.5e6}
 
 def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
     """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
