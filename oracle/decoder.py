@@ -16,7 +16,9 @@ library.
 Pinned by tests/test_oracle_decoder.py: closed forms (RoPE angle, RMSNorm of a
 constant vector, SiLU identity), invariants (cached == uncached, causality,
 relative-position property), library routines (scaled_dot_product_attention,
-and the whole forward against an independent library LLaMA implementation).
+and the whole forward against an independent library LLaMA implementation);
+the bf16 cache option by its defining properties (no effect on values that bf16
+holds exactly, a bounded effect otherwise, the plain result when switched off).
 """
 from __future__ import annotations
 
@@ -89,13 +91,25 @@ def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, q_positions: to
 
 
 class Decoder:
-    def __init__(self, shape, weights: dict, dtype=torch.float64):
+    def __init__(self, shape, weights: dict, dtype=torch.float64, kv_dtype=None):
         """`shape`: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim,
         d_ffn, vocab, rope_theta, rms_eps.  `weights`: name -> tensor, matrices
-        stored [out, in]."""
+        stored [out, in].
+
+        `kv_dtype`: storage type of the KV cache.  None keeps keys and values at the compute
+        dtype (the plain definition).  The paper does not say how the cache is stored; the
+        workloads fix a bf16 cache, and with kv_dtype=torch.bfloat16 every key (after the rotary
+        embedding) and value is rounded to bf16 (round to nearest even, from fp32) at the moment
+        it enters the cache, the rows of the current call included; everything else is unchanged."""
         self.s = shape
         self.w = weights
         self.dtype = dtype
+        self.kv_dtype = kv_dtype
+
+    def _stored(self, t: torch.Tensor) -> torch.Tensor:
+        if self.kv_dtype is None:
+            return t
+        return t.to(torch.float32).to(self.kv_dtype).to(self.dtype)
 
     def _w(self, name: str) -> torch.Tensor:
         return self.w[name].to(self.dtype)
@@ -116,7 +130,8 @@ class Decoder:
             k = (h @ self._w(f"l{l}.wk").T).view(T, s.n_kv_heads, s.head_dim)
             v = (h @ self._w(f"l{l}.wv").T).view(T, s.n_kv_heads, s.head_dim)
             q = rope(q, pos, s.rope_theta)
-            k = rope(k, pos, s.rope_theta)
+            k = self._stored(rope(k, pos, s.rope_theta))
+            v = self._stored(v)
             cache.k[l] = k if cache.k[l] is None else torch.cat([cache.k[l], k], dim=0)
             cache.v[l] = v if cache.v[l] is None else torch.cat([cache.v[l], v], dim=0)
             a = attention(q, cache.k[l], cache.v[l], pos).reshape(T, -1)

@@ -164,3 +164,38 @@ def test_float32_mode_close_to_float64():
     toks = [5, 9, 9, 1, 33, 7, 2, 60]
     a, b = d64.forward(toks, d64.new_cache()), d32.forward(toks, d32.new_cache())
     assert b.dtype == torch.float32 and float((a - b.double()).abs().max()) < 1e-4
+
+
+# ---- bf16 storage of the KV cache (fixed by the workloads, not by the paper) ----
+def _is_bf16_valued(t: torch.Tensor) -> bool:
+    return bool(torch.equal(t.to(torch.float32).to(torch.bfloat16).to(t.dtype), t))
+
+
+def test_bf16_cache_option_stores_bf16_values_and_changes_nothing_else():
+    dec, w = small_model()
+    dec16 = Decoder(SMALL, w, torch.float64, kv_dtype=torch.bfloat16)
+    toks = [3, 17, 5, 40, 9, 22]
+    c0, c1 = dec.new_cache(), dec16.new_cache()
+    l0, l1 = dec.forward(toks, c0), dec16.forward(toks, c1)
+    for l in range(SMALL.n_layers):
+        assert _is_bf16_valued(c1.k[l]) and _is_bf16_valued(c1.v[l])
+        assert not _is_bf16_valued(c0.k[l])                       # the plain cache keeps full precision
+    # layer 0 sees the same inputs in both runs: its stored keys are the plain keys, rounded
+    assert torch.equal(c1.k[0], c0.k[0].to(torch.float32).to(torch.bfloat16).to(torch.float64))
+    assert torch.equal(c1.v[0], c0.v[0].to(torch.float32).to(torch.bfloat16).to(torch.float64))
+    # a perturbation of relative size 2^-9 per cached element: small but not zero
+    d = float((l0 - l1).abs().max())
+    assert 0.0 < d < 0.05 * float(l0.abs().max())
+    # switched off it is the plain forward
+    assert torch.equal(Decoder(SMALL, w, torch.float64, kv_dtype=None).forward(toks, dec.new_cache()), l0)
+
+
+def test_bf16_cache_incremental_equals_full():
+    _, w = small_model()
+    dec16 = Decoder(SMALL, w, torch.float64, kv_dtype=torch.bfloat16)
+    toks = [1, 2, 3, 4, 5, 6, 7]
+    full = dec16.forward(toks, dec16.new_cache())
+    c = dec16.new_cache()
+    a = dec16.forward(toks[:4], c)
+    b = dec16.forward(toks[4:], c)
+    assert torch.allclose(torch.cat([a, b]), full, atol=1e-12, rtol=0)
