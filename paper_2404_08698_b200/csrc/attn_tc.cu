@@ -11,12 +11,12 @@
 // terms each (hi rows then lo rows of the N operand, N = 2 x 8 x G), so only the cache's own bf16
 // rounding is left; the two halves of an accumulator are added when it is read back.
 //
-// The kernel is persistent: one CTA per SM holds up to four independent "slots" (a warpgroup of
+// The kernel is persistent: one CTA per SM holds up to five independent "slots" (a warpgroup of
 // 128 threads with its own 32 KB page buffer, operand staging and tensor-memory columns), and a
 // slot walks through its share of the items.  The page buffer first receives the K page; as soon as
 // the first product has consumed it the V^T page is requested into the same buffer and lands while
-// the softmax runs; after the second product the next item's K page follows.  With four slots per
-// SM every SM keeps several page copies in flight, and at the context lengths of interest each slot
+// the softmax runs; after the second product the next item's K page follows.  With four or five slots
+// per SM every SM keeps several page copies in flight, and at the context lengths of interest each slot
 // has one or two items.
 // Thread t of a slot owns tensor-memory lane t: key t of the page after the first product, output
 // dimension t after the second.  The softmax over the page's keys is a reduction across threads
@@ -52,13 +52,13 @@ __device__ __forceinline__ int b_operand_offset(int n, int k) {
     return (k >> 6) * (N * 128) + (n >> 3) * 1024 + (n & 7) * 128 + ((((kk >> 3) ^ (n & 7))) << 4) + (kk & 7) * 2;
 }
 
-// Slots per CTA for G query heads per kv head: what fits in shared memory and tensor memory.
-template <int G> struct AttnCfg {
+// S slots per CTA for G query heads per kv head (bounded by shared memory and tensor memory).
+template <int G, int S> struct AttnCfg {
     static constexpr int Q = 8 * G;                      // query vectors: 8 rows x G heads of the group
     static constexpr int N = 2 * Q;                      // MMA N: hi terms then lo terms
     static constexpr int B_BYTES = N * 256;              // one N-row operand (two 64-column tiles)
     static constexpr int SLOT_BYTES = 2 * PAGE_ATOM + 2 * B_BYTES;       // page buffer (K, then V), Q operand, P operand
-    static constexpr int SLOTS = (G <= 2) ? 4 : (G == 4) ? 3 : 2;       // G = 1 would fit five; four measured faster
+    static constexpr int SLOTS = S;
     static constexpr int THREADS = SLOTS * 128;
     static constexpr int TMEM_NEED = SLOTS * N;          // per slot N columns: S^T, then O^T in the same columns
     static constexpr int TMEM_COLS = TMEM_NEED <= 32 ? 32 : TMEM_NEED <= 64 ? 64 : TMEM_NEED <= 128 ? 128 : TMEM_NEED <= 256 ? 256 : 512;
@@ -69,13 +69,13 @@ __device__ __forceinline__ void slot_bar(int slot) { asm volatile("bar.sync %0, 
 
 struct AttnItem { int c, kvh, r0, pos_lo, seq; };
 
-template <int G>
-__global__ void __launch_bounds__(AttnCfg<G>::THREADS, 1)
+template <int G, int S>
+__global__ void __launch_bounds__(AttnCfg<G, S>::THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const bf16* __restrict__ q_hi,
                const bf16* __restrict__ q_lo, const int* __restrict__ page_table, int pages_per_seq, const int* __restrict__ row_pos,
                const int* __restrict__ row_seq, int Hq, int Hkv, int layer_row0, int chunks, int n_items, float* __restrict__ pm,
                float* __restrict__ pl, float* __restrict__ po, int* err) {
-    typedef AttnCfg<G> Cfg;
+    typedef AttnCfg<G, S> Cfg;
     constexpr int Q = Cfg::Q, N = Cfg::N, SLOTS = Cfg::SLOTS;
     extern __shared__ __align__(1024) unsigned char attn_tc_smem[];
     __shared__ uint64_t bar_k[SLOTS], bar_v[SLOTS], bar_s[SLOTS], bar_o[SLOTS];
@@ -292,21 +292,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     }
 }
 
-template <int G>
+template <int G, int S>
 anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int chunks) {
-    typedef AttnCfg<G> Cfg;
+    typedef AttnCfg<G, S> Cfg;
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
     static bool attr_set = false;
     if (!attr_set) {
-        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
         attr_set = true;
     }
     const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
     const int n_items = chunks * c.n_kv_heads * (rows / ANPD_ROWS);
     const int grid = std::min(m->num_sms, n_items);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_tc_kernel<G>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
+           (launch_k(attn_tc_kernel<G, S>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
                      kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
                      ws.attn_l, ws.attn_o, ws.gemm_err)));
     return ANPD_OK;
@@ -316,11 +316,15 @@ anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int 
 
 anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos) {
     const int chunks = max_pos / KV_PAGE + 1;
+    const int n_items = chunks * m->cfg.n_kv_heads * (rows / ANPD_ROWS);
     switch (m->cfg.n_q_heads / m->cfg.n_kv_heads) {
-        case 1: return launch_attn_tc<1>(m, kv, layer, rows, chunks);
-        case 2: return launch_attn_tc<2>(m, kv, layer, rows, chunks);
-        case 4: return launch_attn_tc<4>(m, kv, layer, rows, chunks);
-        case 8: return launch_attn_tc<8>(m, kv, layer, rows, chunks);
+        // one query head per kv head fits five slots; while every item finds a slot with four, four are faster
+        // (measured at the 7B shape: 1.2 % of the step at 17 pages; with 33 pages five slots win by 2.4 %)
+        case 1: return n_items <= 4 * m->num_sms ? launch_attn_tc<1, 4>(m, kv, layer, rows, chunks)
+                                                 : launch_attn_tc<1, 5>(m, kv, layer, rows, chunks);
+        case 2: return launch_attn_tc<2, 4>(m, kv, layer, rows, chunks);
+        case 4: return launch_attn_tc<4, 3>(m, kv, layer, rows, chunks);
+        case 8: return launch_attn_tc<8, 2>(m, kv, layer, rows, chunks);
     }
     return ANPD_ERR_ARG;
 }
