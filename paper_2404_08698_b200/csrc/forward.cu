@@ -23,18 +23,6 @@ __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-// Sum over a 256-thread block in a fixed order (xor-shuffle tree per warp, then across warps).
-__device__ __forceinline__ float block_sum_256(float v, float* red /*[8]*/) {
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    float t = (threadIdx.x & 31) < 8 ? red[threadIdx.x & 31] : 0.0f;
-    for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    t = __shfl_sync(0xffffffffu, t, 0);
-    __syncthreads();
-    return t;
-}
-
 // ---------------------------------------------------------------------------------------------
 // row plans
 // ---------------------------------------------------------------------------------------------
