@@ -175,7 +175,9 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
                                        bf16* __restrict__ q_lo, bf16* __restrict__ kpool_l, bf16* __restrict__ vpool_l) {
     pdl_trigger();
     pdl_wait();
-    const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
+    // a block covers blockDim.x / (hd / 2) consecutive heads of one row
+    const int half = hd >> 1, row = blockIdx.x, head = blockIdx.y * (blockDim.x / half) + threadIdx.x / half, i = threadIdx.x % half;
+    if (head >= Hq + 2 * Hkv) return;
     const float* pr = part + (size_t)row * ld_part + (size_t)head * hd;
     float a = 0.0f, b = 0.0f;
     const int ns = seg_count[(head * hd + i) >> 7];      // a head never straddles a 128-column tile
@@ -504,6 +506,59 @@ __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* _
     }
 }
 
+// The same for many rows (prefill passes), shaped for throughput: four warps per (row, q head), a lane owns hd/32
+// consecutive dimensions and fetches them in one load per page.  Slices, page order within a slice, the order of the
+// slices and the total weight are those of attn_combine_kernel, so the results are the same bits.
+template <int VEC>
+__global__ void __launch_bounds__(32 * COMBINE_SLICES) attn_combine_wide_kernel(const float* __restrict__ pm, const float* __restrict__ pl,
+                                                                               const float* __restrict__ po, const int* __restrict__ row_pos,
+                                                                               int Hq, int pages_per_seq, bf16* __restrict__ ao_hi,
+                                                                               bf16* __restrict__ ao_lo) {
+    pdl_trigger();
+    pdl_wait();
+    constexpr int hd = 32 * VEC;
+    __shared__ float s_m[COMBINE_MAX_PAGES];
+    __shared__ float s_l[COMBINE_MAX_PAGES];
+    __shared__ float s_o[COMBINE_SLICES][hd];
+    const int row = blockIdx.x, head = blockIdx.y;
+    const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+    const int nc = min(row_pos[row] / KV_PAGE + 1, COMBINE_MAX_PAGES);
+    const size_t base = ((size_t)row * Hq + head) * pages_per_seq;
+    for (int c = threadIdx.x; c < nc; c += blockDim.x) { s_m[c] = pm[base + c]; s_l[c] = pl[base + c]; }
+    __syncthreads();
+    float M = -CUDART_INF_F;
+    for (int c = 0; c < nc; ++c) M = fmaxf(M, s_m[c]);
+    float L = 0.0f;
+    for (int c = 0; c < nc; ++c) L = fmaf(s_l[c], exp2f(s_m[c] - M), L);       // partial maxima are in the base-2 domain
+    float o[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) o[e] = 0.0f;
+    for (int c = slice; c < nc; c += COMBINE_SLICES) {
+        const float w = exp2f(s_m[c] - M);
+        const float* src = po + (base + c) * hd + lane * VEC;
+        float v[VEC];
+        if (VEC == 4) { const float4 t = *(const float4*)src; v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+        else { const float2 t = *(const float2*)src; v[0] = t.x; v[1] = t.y; }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) o[e] = fmaf(v[e], w, o[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) s_o[slice][lane * VEC + e] = o[e];
+    __syncthreads();
+    if (slice == 0) {
+        const size_t out = (size_t)row * Hq * hd + head * hd + lane * VEC;
+        bf16 h[VEC], l[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            float t = s_o[0][lane * VEC + e];
+            for (int k = 1; k < COMBINE_SLICES; ++k) t += s_o[k][lane * VEC + e];
+            split_bf16(t / L, h[e], l[e]);
+        }
+        if (VEC == 4) { *(uint2*)(ao_hi + out) = *(const uint2*)h; *(uint2*)(ao_lo + out) = *(const uint2*)l; }
+        else { *(uint32_t*)(ao_hi + out) = *(const uint32_t*)h; *(uint32_t*)(ao_lo + out) = *(const uint32_t*)l; }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // SwiGLU epilogue of the gate/up projection
 // ---------------------------------------------------------------------------------------------
@@ -523,6 +578,27 @@ __global__ void swiglu_kernel(const float* __restrict__ part, const int* __restr
     split_bf16(v, hi, lo);
     act_hi[(size_t)row * F + j] = hi;
     act_lo[(size_t)row * F + j] = lo;
+}
+
+// The same for many rows (prefill passes): a thread owns four consecutive features, so the partial sums come in
+// 16-byte loads.  Per element the arithmetic is that of swiglu_kernel, in the same order.
+__global__ void swiglu_wide_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride, int ld_part, int F,
+                                   bf16* __restrict__ act_hi, bf16* __restrict__ act_lo) {
+    pdl_trigger();
+    pdl_wait();
+    const int row = blockIdx.y, j = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
+    if (j >= F) return;
+    const float* pr = part + (size_t)row * ld_part;
+    float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), u4 = g4;
+    const int ng = seg_count[j >> 7], nu = seg_count[(F + j) >> 7];
+    for (int s = 0; s < ng; ++s) { const float4 p = *(const float4*)(pr + s * split_stride + j); g4.x += p.x; g4.y += p.y; g4.z += p.z; g4.w += p.w; }
+    for (int s = 0; s < nu; ++s) { const float4 p = *(const float4*)(pr + s * split_stride + F + j); u4.x += p.x; u4.y += p.y; u4.z += p.z; u4.w += p.w; }
+    const float gte[4] = {g4.x, g4.y, g4.z, g4.w}, up[4] = {u4.x, u4.y, u4.z, u4.w};
+    bf16 hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) split_bf16(gte[e] / (1.0f + expf(-gte[e])) * up[e], hi[e], lo[e]);
+    *(uint2*)(act_hi + (size_t)row * F + j) = *(const uint2*)hi;
+    *(uint2*)(act_lo + (size_t)row * F + j) = *(const uint2*)lo;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -718,7 +794,10 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
                          kv->vpool + layer * layer_elems, kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads,
                          c.n_kv_heads, ws.attn_m, ws.attn_l, ws.attn_o)));
     }
-    LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
+    if (rows >= 64) LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
+           (launch_k(attn_combine_wide_kernel<HD / 32>, dim3(rows, c.n_q_heads), 32 * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o,
+                     ws.row_pos, c.n_q_heads, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
+    else LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
     return ANPD_OK;
@@ -776,11 +855,13 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
 
     LAUNCH(pf, st, KC_OTHER, 0, (launch_k(embed_norm_kernel, rows, NORM_THREADS, 0, st, m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
                                                                       ws.x, ws.h_hi, ws.h_lo)));
+    const bool many_rows = rows >= 64;                 // prefill passes: throughput-shaped launches of the small kernels
+    const int rope_hpb = many_rows ? 256 / (hd / 2) : 1;            // heads per block of the rotary kernel
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& w = m->layers[l];
         ANPD_TRY(gemm_enqueue(m, kv, GK_QKV, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
-               (launch_k(qkv_rope_append_kernel, dim3(rows, c.n_q_heads + 2 * c.n_kv_heads), hd / 2, 0, st, 
+               (launch_k(qkv_rope_append_kernel, dim3(rows, (c.n_q_heads + 2 * c.n_kv_heads + rope_hpb - 1) / rope_hpb), rope_hpb * (hd / 2), 0, st, 
                    ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
                    kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, hd, 1.4426950408889634f / sqrtf((float)hd), ws.q_hi,
                    ws.q_lo, kv->kpool + l * layer_elems, kv->vpool + l * layer_elems)));
@@ -791,7 +872,10 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
                (launch_k(resid_norm_kernel, rows, NORM_THREADS, 0, st, ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
                                                        ws.h_hi, ws.h_lo)));
         ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs));
-        LAUNCH(pf, st, KC_OTHER, 0,
+        if (many_rows) LAUNCH(pf, st, KC_OTHER, 0,
+               (launch_k(swiglu_wide_kernel, dim3((F / 4 + 255) / 256, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
+                         ws.act_lo)));
+        else LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(swiglu_kernel, dim3((F + 255) / 256, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
                                                                           ws.act_lo)));
         ANPD_TRY(gemm_enqueue(m, kv, GK_DOWN, l, rows, &segs));
