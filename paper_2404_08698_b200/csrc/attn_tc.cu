@@ -297,10 +297,9 @@ anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int 
     typedef AttnCfg<G, S> Cfg;
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};
+    if (first_call_on_device(attr_set)) {
         CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
-        attr_set = true;
     }
     const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
     const int n_items = chunks * c.n_kv_heads * (rows / ANPD_ROWS);

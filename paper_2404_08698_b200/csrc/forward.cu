@@ -780,10 +780,9 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     const int chunks = max_pos / KV_PAGE + 1;
     const size_t smem = (size_t)KV_PAGE * (HD * 2 + 64) + (size_t)HD * (KV_PAGE * 2 + 64);
     static_assert(4 * 16 * (HD + 4) * sizeof(float) <= (size_t)KV_PAGE * (HD * 2 + 64), "merge buffer must fit in the K staging area");
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};
+    if (first_call_on_device(attr_set)) {
         CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set = true;
     }
     if (HD == 128 && kv->attn_tc) {
         ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos));

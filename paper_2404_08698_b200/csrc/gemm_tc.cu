@@ -323,10 +323,9 @@ int gemm_smem_bytes(int NB, int* stages_out) {
 anpd_status gemm_tc_enqueue(const GemmPlan& plan, const bf16* w_blocks, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
                             int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,
                             Profiler* prof) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};
+    if (first_call_on_device(attr_set)) {
         CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-        attr_set = true;
     }
     GemmArgs g;
     g.part = part; g.seg_stride = seg_stride; g.ld_part = ld_part;

@@ -30,6 +30,16 @@ void anpd_note_cuda_error(cudaError_t e, const char* file, int line);
         if (s__ != ANPD_OK) return s__;      \
     } while (0)
 
+// One-time per-device set-up inside a launch helper (function attributes are per device): true the first time it
+// is called for the current device with this flag array, which the caller keeps as a function-local static.
+inline bool first_call_on_device(bool (&done)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+    if (done[dev]) return false;
+    done[dev] = true;
+    return true;
+}
+
 // ---------------------------------------------------------------------------------------------
 // launch accounting + optional per-class timing
 // ---------------------------------------------------------------------------------------------
