@@ -128,6 +128,50 @@ def test_c3_attention_kernels_agree_at_bench_context_length(A, c3, monkeypatch):
     assert float(np.abs(outs[0][1] - outs[1][1]).max()) <= 1e-2
 
 
+def _short_prompt_logits_check(A, wl, n_prompt, tol):
+    """Model of workload `wl` at full size: prefill `n_prompt` tokens, one 8-row verify step, logits against the
+    oracle with the bf16 cache; returns (max-abs error, the oracle's logit standard deviation)."""
+    w = make_weights(wl.shape, wl.weight_seed, True, device="cuda")
+    torch.cuda.synchronize()
+    m = gpu_model(A, wl.shape, w, new_stream())
+    w_cpu = {k: v.cpu() for k, v in w.items()}
+    del w
+    torch.cuda.empty_cache()
+    prompt = make_prompts(wl)[0][:n_prompt].tolist()
+    draft = [int(t) for t in make_prompts(wl)[0][n_prompt + 8:n_prompt + 15]]
+    kv = A.anpd_kv_create(m, 256)
+    try:
+        first = A.anpd_prefill(m, kv, prompt)
+        got = A.anpd_verify_logits(m, kv, first, draft, wl.shape.vocab)
+    finally:
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(m)
+    dec = Decoder(wl.shape, w_cpu, torch.float64, kv_dtype=torch.bfloat16)
+    cache = dec.new_cache()
+    lp = dec.forward(prompt, cache)
+    if top2_margin(lp[-1]) > 2 * tol:
+        assert first == argmax_lowest(lp[-1])
+    want = dec.forward([first] + draft, cache)
+    diff = torch.from_numpy(got).double() - want
+    for r in range(want.shape[0]):
+        if top2_margin(want[r]) > 2 * tol:
+            assert int(np.argmax(got[r])) == argmax_lowest(want[r])
+    return float(diff.abs().max()), float(diff.pow(2).mean().sqrt())
+
+
+def test_c2_shape_grouped_query_heads_against_oracle(A):
+    """1.1B shape: 22 layers, 32 query heads on 4 kv heads of dimension 64 (the mma.sync attention kernel with 8 query
+    heads per kv head), d_ffn 5632; 40-token prompt."""
+    err, rms = _short_prompt_logits_check(A, WORKLOADS["C2"], 40, FULLSIZE_TOL)
+    assert err <= FULLSIZE_TOL and rms <= 1e-2, (err, rms)
+
+
+def test_c5_shape_single_sequence_against_oracle(A):
+    """13B shape: 40 layers x 5120, 40 heads of dimension 128, d_ffn 13824 (other stream-K splits than the 7B shape)."""
+    err, rms = _short_prompt_logits_check(A, WORKLOADS["C5"], 10, FULLSIZE_TOL)
+    assert err <= FULLSIZE_TOL and rms <= 1e-2, (err, rms)
+
+
 def test_largest_projection_sampled_against_fp64(A):
     """gate/up projection of the 7B shape [22016 x 4096], 8 rows: 64 sampled output features per row."""
     N, K, rows = 22016, 4096, 8
