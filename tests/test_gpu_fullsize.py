@@ -172,6 +172,38 @@ def test_c5_shape_single_sequence_against_oracle(A):
     assert err <= FULLSIZE_TOL and rms <= 1e-2, (err, rms)
 
 
+def test_c5_batch_of_eight_equals_greedy_and_independent_runs(A):
+    """13B shape, 8 sequences in one step (64 rows per launch, per-sequence tables and KV pages): the batched ANPD
+    streams equal the batched greedy streams and the streams of sequences run on their own."""
+    wl = WORKLOADS["C5"]
+    w = make_weights(wl.shape, wl.weight_seed, True, device="cuda")
+    torch.cuda.synchronize()
+    st = new_stream()
+    m = gpu_model(A, wl.shape, w, st)
+    del w
+    torch.cuda.empty_cache()
+    B, plen, M = wl.batch, 300, 20
+    prompts = np.stack([p[:plen] for p in make_prompts(wl)])
+    kvb = A.anpd_kv_create(m, 512, B)
+    kv1 = A.anpd_kv_create(m, 512, 1)
+    ctxs = [A.anpd_ngram_create(wl.n_min, wl.n_max, 512, 0, st) for _ in range(B)]
+    try:
+        outs, stats = A.anpd_generate_batch(m, kvb, ctxs, prompts, M, wl.K)
+        greedy, _ = A.anpd_generate_batch(m, kvb, ctxs, prompts, M, 0)
+        assert np.array_equal(outs, greedy)
+        for b in (0, 5):
+            single, st1 = A.anpd_generate(m, kv1, ctxs[0], prompts[b], M, wl.K)
+            assert np.array_equal(single, outs[b]), b
+            for k in ("steps", "drafted", "accepted", "generated"):
+                assert st1[k] == stats[b][k], (b, k)
+    finally:
+        for c in ctxs:
+            A.anpd_ngram_destroy(c)
+        A.anpd_kv_destroy(kv1)
+        A.anpd_kv_destroy(kvb)
+        A.anpd_model_destroy(m)
+
+
 def test_largest_projection_sampled_against_fp64(A):
     """gate/up projection of the 7B shape [22016 x 4096], 8 rows: 64 sampled output features per row."""
     N, K, rows = 22016, 4096, 8
