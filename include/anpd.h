@@ -187,7 +187,8 @@ anpd_status anpd_verify_logits(anpd_model* m, anpd_kv* kv, int32_t last_tok, con
 /* Asynchronous layer under anpd_verify_batch, for timing with events on the model's stream:
  * stage copies the step's inputs for all sequences to the device; enqueue issues the forward,
  * accept and commit; result waits and reads the outcome.  enqueue may be called repeatedly
- * (with anpd_kv_truncate in between) without re-staging. */
+ * without re-staging, but between two enqueues the library must learn the cache lengths again:
+ * either anpd_verify_result, or anpd_kv_truncate for every sequence; otherwise ANPD_ERR_STATE. */
 anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_tok,
                               const int32_t* drafts, const int* draft_len);
 anpd_status anpd_verify_enqueue(anpd_model* m, anpd_kv* kv);

@@ -300,6 +300,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     // the legacy default stream cannot be captured: steps on it are launched one kernel at a time
     kv->use_graphs = std::getenv("ANPD_NO_GRAPH") == nullptr && m->stream != nullptr && m->stream != cudaStreamLegacy;
     kv->h_kv_len.assign(batch, 0);
+    kv->h_len_stale.assign(batch, 0);
     Workspace& ws = kv->ws;
     ws.r_max = std::max(PREFILL_ROWS, batch * ANPD_ROWS);
     ws.n_max_out = (std::max(std::max(m->nqkv, 2 * c.d_ffn), std::max(c.d_model, c.vocab)) + 127) / 128 * 128;
@@ -423,6 +424,7 @@ anpd_status anpd_kv_truncate(anpd_kv* kv, int seq, int len) {
     LAUNCH(&kv->m->prof, kv->m->stream, KC_OTHER, 0, (set_int_kernel<<<1, 1, 0, kv->m->stream>>>(&kv->seq[seq].kv_len, len)));
     CUDA_TRY(cudaGetLastError());
     kv->h_kv_len[seq] = len;
+    kv->h_len_stale[seq] = 0;
     return ANPD_OK;
 }
 
@@ -433,6 +435,7 @@ static anpd_status kv_reset(anpd_kv* kv, const int* stop_at) {
         kv->h_seq[b].active = 1;
         kv->h_seq[b].stop_at = stop_at ? stop_at[b] : 0x7fffffff;
         kv->h_kv_len[b] = 0;
+        kv->h_len_stale[b] = 0;
     }
     CUDA_TRY(cudaMemcpyAsync(kv->seq, kv->h_seq, sizeof(SeqState) * (size_t)kv->batch, cudaMemcpyHostToDevice, kv->m->stream));
     CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
@@ -461,7 +464,7 @@ static anpd_status read_seqs(anpd_kv* kv) {
     CUDA_TRY(cudaMemcpyAsync(kv->h_seq, kv->seq, sizeof(SeqState) * (size_t)kv->batch, cudaMemcpyDeviceToHost, kv->m->stream));
     CUDA_TRY(cudaMemcpyAsync(h_err, kv->ws.gemm_err, sizeof(int), cudaMemcpyDeviceToHost, kv->m->stream));
     CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
-    for (int b = 0; b < kv->batch; ++b) kv->h_kv_len[b] = kv->h_seq[b].kv_len;
+    for (int b = 0; b < kv->batch; ++b) { kv->h_kv_len[b] = kv->h_seq[b].kv_len; kv->h_len_stale[b] = 0; }
     if (*h_err != 0) {
         std::snprintf(g_last_error, sizeof(g_last_error), "a GEMM kernel gave up waiting (code %d)", *h_err);
         return ANPD_ERR_CUDA;
@@ -524,6 +527,8 @@ anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_to
 static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K = -1) {
     int max_pos = 0;
     for (int b = 0; b < kv->batch; ++b) {
+        // the attention grid is sized from the host's copy of the lengths: it must not be behind the device
+        if (kv->h_len_stale[b]) return ANPD_ERR_STATE;
         if (kv->h_kv_len[b] + ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
         max_pos = std::max(max_pos, kv->h_kv_len[b] + ANPD_ROWS - 1);
     }
@@ -542,6 +547,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
         if (m->prof.on) g_use_pdl = false;            // per-launch timing needs kernels that do not overlap
         const anpd_status rc = enqueue();
         g_use_pdl = pdl;
+        if (rc == ANPD_OK && mode == ACCEPT_COMMIT) std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1);
         return rc;
     }
     const uint64_t key = (uint64_t)(max_pos / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)mode << 24) |
@@ -553,7 +559,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
         if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
             cudaGetLastError();
             kv->use_graphs = false;
-            return enqueue();
+            { const anpd_status r2 = enqueue(); if (r2 == ANPD_OK && mode == ACCEPT_COMMIT) std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1); return r2; }
         }
         const anpd_status rc = enqueue();
         const cudaError_t ce = cudaStreamEndCapture(st, &graph);
@@ -564,13 +570,14 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
             cudaGetLastError();
             if (graph) cudaGraphDestroy(graph);
             kv->use_graphs = false;                   // fall back to plain launches for good
-            return enqueue();
+            { const anpd_status r2 = enqueue(); if (r2 == ANPD_OK && mode == ACCEPT_COMMIT) std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1); return r2; }
         }
         cudaGraphDestroy(graph);
         it = kv->graphs.emplace(key, sg).first;
     }
     CUDA_TRY(cudaGraphLaunch(it->second.exec, st));
     g_launch_count += it->second.launches;
+    if (mode == ACCEPT_COMMIT) std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1);
     return ANPD_OK;
 }
 

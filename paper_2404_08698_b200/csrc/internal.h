@@ -244,6 +244,7 @@ struct anpd_kv {
     NgramDev* d_ctxs;                 // device [batch]: descriptors of the sequences' n-gram contexts
     int* h_small;                     // pinned, a few ints
     std::vector<int> h_kv_len;        // host mirror of the sequences' lengths
+    std::vector<char> h_len_stale;    // a committing step was enqueued and its outcome not read yet: the mirror is behind
     Workspace ws;
     void* slab;
     size_t slab_bytes;

@@ -201,6 +201,18 @@ def test_verify_error_paths(A, c1):
     with pytest.raises(A.AnpdError) as e:
         A.anpd_prefill(c1.m, c1.kv, [1, 2, 3])                         # cache not empty
     assert e.value.status == A.ERR_STATE
+    # a second committing step may not be enqueued before the outcome of the first is known to the host
+    A.anpd_verify_stage(c1.m, c1.kv, [5], [[6, 7]])
+    A.anpd_verify_enqueue(c1.m, c1.kv)
+    with pytest.raises(A.AnpdError) as e:
+        A.anpd_verify_enqueue(c1.m, c1.kv)
+    assert e.value.status == A.ERR_STATE
+    A.anpd_kv_truncate(c1.kv, 0, 3)                                    # tells the library the length again
+    A.anpd_verify_enqueue(c1.m, c1.kv)
+    acc, nxt = A.anpd_verify_result(c1.m, c1.kv)
+    assert 0 <= acc[0] <= 2
+    A.anpd_verify_enqueue(c1.m, c1.kv)                                 # allowed again after the result was read
+    A.anpd_verify_result(c1.m, c1.kv)
     with pytest.raises(A.AnpdError) as e:
         A.anpd_kv_truncate(c1.kv, 0, 10)                               # cannot grow
     assert e.value.status == A.ERR_RANGE
