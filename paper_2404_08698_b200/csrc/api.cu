@@ -466,7 +466,7 @@ static anpd_status read_seqs(anpd_kv* kv) {
     CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
     for (int b = 0; b < kv->batch; ++b) { kv->h_kv_len[b] = kv->h_seq[b].kv_len; kv->h_len_stale[b] = 0; }
     if (*h_err != 0) {
-        std::snprintf(g_last_error, sizeof(g_last_error), "a GEMM kernel gave up waiting (code %d)", *h_err);
+        std::snprintf(g_last_error, sizeof(g_last_error), "a kernel gave up waiting on a barrier (code %d: 201 GEMM, 202 attention)", *h_err);
         return ANPD_ERR_CUDA;
     }
     return ANPD_OK;
