@@ -14,7 +14,14 @@
  *   - Every function returns an anpd_status: 0 on success, negative on failure.  Nothing
  *     aborts or throws.  On failure the caller's output arguments are left untouched.
  *   - Handles (anpd_model, anpd_kv, anpd_ngram) are opaque, owned by the library and
- *     released by the matching *_destroy.  One handle is used by one thread at a time.
+ *     released by the matching *_destroy.  One handle is used by one thread at a time; a kv or
+ *     ngram handle belongs with its model, so one model and everything created for it stay on
+ *     one thread at a time.  Different models may be used from different threads: the library
+ *     keeps no mutable state outside the handles except the launch counter (atomic) and the text
+ *     of the calling thread's last CUDA failure (thread-local).
+ *   - A model is laid out for the device that was current when it was created (the weight
+ *     blocks are ordered for that device's SM count).  Using its handles while another device
+ *     is current returns ANPD_ERR_STATE.
  *   - Array arguments are caller-owned HOST memory unless the parameter comment says
  *     "device"; they are only read or written during the call.
  *   - All device work of a model, and of the kv / ngram handles used with it, is issued on
@@ -198,9 +205,11 @@ anpd_status anpd_verify_result(anpd_model* m, anpd_kv* kv, int* accepted_len, in
  * prompt -> Initialize + prefill -> repeat {commit, Update, draft K, verify, accept} until
  * max_new tokens are out; the result is cut to max_new.  K == 0 is plain greedy decoding
  * through the same kernels at the same row count, so the two token streams are bit-identical.
- * kv and ctx are reset first.  out: int32[max_new]; *n_out = tokens written (max_new unless the
- * context or the cache fills up, which returns ANPD_ERR_CAPACITY after writing what fits).
- * stats may be NULL. */
+ * kv and ctx are reset first.  out: int32[max_new]; *n_out = max_new on success.  Capacity is
+ * checked before any work: the context needs prompt_len + max_new + 9 <= max_ctx and the cache
+ * prompt_len + max_new + 16 <= max_len (the loop may overshoot max_new by up to K tokens and
+ * every step writes 8 rows); otherwise ANPD_ERR_CAPACITY is returned with out and n_out
+ * untouched.  stats may be NULL. */
 anpd_status anpd_generate(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const int32_t* prompt,
                           int prompt_len, int max_new, int K, int32_t* out, int* n_out,
                           anpd_stats* stats);
@@ -245,7 +254,8 @@ anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a
  * The array is shared by all calls on a device and keeps the previous call's contents; the call
  * clears what must start at zero itself.  Calls that overlap on the GPU (two streams, two threads)
  * race on it: issue them one after the other.  The first call on a device looks up the array's
- * device address; make that first call before any stream capture begins. */
+ * device address; make that first call before any stream capture begins.  Every call waits for
+ * its work on cuda_stream and reads a status word back before it returns. */
 anpd_status anpd_gemm_static(const uint16_t* w_bf16_dev, int N, int K, const float* a_dev, int rows,
                              float* out_dev, void* cuda_stream);
 

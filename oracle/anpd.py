@@ -10,7 +10,7 @@ cache has `.length` and `.truncate(n)`: the decoder oracle, or a scripted
 stand-in in tests.  Only tests, the smoke check and the benchmark's CPU
 baseline may import this file.
 
-Readings (the design doc lists them):
+Readings taken where Algorithm 1 is ambiguous:
   * drafts[1] of a step is the already confirmed token; the model's prediction
     after consuming drafts[1..i] is compared with drafts[i+1].
   * after `a` accepted drafts the next confirmed token is the prediction that

@@ -3,7 +3,7 @@
 The "LLM" of Algorithm 1: LLM(prompt) (prefill) and LLM(drafts) (one forward
 over the K+1 tokens of a step against the KV cache, Section 3.1 "Verification").
 The paper names only the model family; the internals below are the published
-LLaMA architecture with the conventions the design doc lists (RMSNorm, rotary
+LLaMA architecture (RMSNorm with eps under the root, rotary
 embedding with rotate-half pairing, no biases, SwiGLU, untied LM head).
 
 Plain torch CPU ops in a chosen dtype (float64 by default; float32 on request),
@@ -91,7 +91,7 @@ def attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, q_positions: to
 
 
 class Decoder:
-    def __init__(self, shape, weights: dict, dtype=torch.float64, kv_dtype=None):
+    def __init__(self, shape, weights: dict, dtype=torch.float64, kv_dtype=None, keep_cast: bool = False):
         """`shape`: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim,
         d_ffn, vocab, rope_theta, rms_eps.  `weights`: name -> tensor, matrices
         stored [out, in].
@@ -100,11 +100,15 @@ class Decoder:
         dtype (the plain definition).  The paper does not say how the cache is stored; the
         workloads fix a bf16 cache, and with kv_dtype=torch.bfloat16 every key (after the rotary
         embedding) and value is rounded to bf16 (round to nearest even, from fp32) at the moment
-        it enters the cache, the rows of the current call included; everything else is unchanged."""
+        it enters the cache, the rows of the current call included; everything else is unchanged.
+
+        `keep_cast`: keep each weight's copy in the compute dtype after its first use instead of
+        casting it again in every forward (same values, more memory: used when the oracle is timed)."""
         self.s = shape
         self.w = weights
         self.dtype = dtype
         self.kv_dtype = kv_dtype
+        self._cast: dict[str, torch.Tensor] | None = {} if keep_cast else None
 
     def _stored(self, t: torch.Tensor) -> torch.Tensor:
         if self.kv_dtype is None:
@@ -112,7 +116,11 @@ class Decoder:
         return t.to(torch.float32).to(self.kv_dtype).to(self.dtype)
 
     def _w(self, name: str) -> torch.Tensor:
-        return self.w[name].to(self.dtype)
+        if self._cast is None:
+            return self.w[name].to(self.dtype)
+        if name not in self._cast:
+            self._cast[name] = self.w[name].to(self.dtype)
+        return self._cast[name]
 
     def new_cache(self) -> KVCache:
         return KVCache(self.s.n_layers)

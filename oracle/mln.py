@@ -6,7 +6,7 @@ multi-level back-off (Section 3.2 and Algorithm 2), written with Python dicts
 over token-id tuples.  Only tests, the smoke check and the benchmark's CPU
 baseline may import this file; it shares no code with the CUDA library.
 
-Readings taken where the paper is silent (all listed in the design doc):
+Readings taken where the paper is silent:
   * Query returns the most probable successor under the frequency counts of
     Eq. 1, i.e. the successor with the largest count; equal counts are broken
     in favour of the successor seen most recently ("max-count" policy).  A
@@ -71,14 +71,10 @@ class MLN:
         return max(cands.items(), key=lambda kv: kv[1][1])[0]
 
     def query(self, ctx) -> int | None:
-        """Algorithm 2: from n = N down to the lowest level, first level that answers wins."""
-        n = self.n_max
-        while n >= self.n_min:
-            pred = self.query_level(n, ctx)
-            if pred is not None:
-                return pred
-            n -= 1
-        return None
+        """Multi-level back-off (Section 3.2, Algorithm 2): the answer of the highest level
+        n in [n_min, n_max] whose table knows the last n-1 tokens of `ctx`; None if no level does."""
+        answers = (self.query_level(n, ctx) for n in range(self.n_max, self.n_min - 1, -1))
+        return next((a for a in answers if a is not None), None)
 
     def draft(self, K: int) -> list[int]:
         """Drafting stage (Section 3.1, Algorithm 1's inner loop): K chained queries,

@@ -10,9 +10,11 @@
 
 typedef __nv_bfloat16 bf16;
 
-long long g_launch_count = 0;
-bool g_use_pdl = std::getenv("ANPD_NO_PDL") == nullptr;
-static char g_last_error[256] = "";
+std::atomic<long long> g_launch_count{0};
+const bool g_use_pdl = std::getenv("ANPD_NO_PDL") == nullptr;
+thread_local bool t_no_pdl = false;
+// text of the calling thread's last CUDA failure (anpd_status_string(ANPD_ERR_CUDA) returns it)
+static thread_local char g_last_error[256] = "";
 
 void anpd_note_cuda_error(cudaError_t e, const char* file, int line) {
     std::snprintf(g_last_error, sizeof(g_last_error), "%s at %s:%d", cudaGetErrorString(e), file, line);
@@ -101,6 +103,14 @@ anpd_status upload(void* dst, const void* src, size_t n, bool as_bf16, bool src_
     return ANPD_OK;
 }
 
+// The model's weight blocks are ordered for the SM count of the device it was created on, and its
+// memory lives there: refuse to run with another device current.
+anpd_status check_device(const anpd_model* m) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return ANPD_ERR_CUDA; }
+    return dev == m->device ? ANPD_OK : ANPD_ERR_STATE;
+}
+
 bool have_device() {
     int n = 0;
     if (cudaGetDeviceCount(&n) != cudaSuccess || n == 0) { cudaGetLastError(); return false; }
@@ -154,9 +164,7 @@ const char* anpd_status_string(anpd_status s) {
 }
 
 long long anpd_launch_count(int reset) {
-    const long long v = g_launch_count;
-    if (reset) g_launch_count = 0;
-    return v;
+    return reset ? g_launch_count.exchange(0) : g_launch_count.load();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -196,6 +204,7 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
             cudaGetLastError(); delete m; return ANPD_ERR_CUDA;
         }
         m->num_sms = sms;
+        m->device = dev;
         const int shapes[GK_COUNT][2] = {{m->nqkv, c.d_model}, {c.d_model, m->dq}, {2 * c.d_ffn, c.d_model}, {c.d_model, c.d_ffn},
                                          {c.vocab, c.d_model}};
         for (int k = 0; k < GK_COUNT; ++k) gemm_make_plan(&m->plan[k], shapes[k][0], shapes[k][1], sms);
@@ -481,6 +490,7 @@ static anpd_status seq_error_status(const SeqState& s) {
 
 anpd_status anpd_prefill(anpd_model* m, anpd_kv* kv, int seq, const int32_t* prompt, int prompt_len, int32_t* first_tok) {
     if (!m || !kv || !prompt || !first_tok || kv->m != m || seq < 0 || seq >= kv->batch || prompt_len < 1) return ANPD_ERR_ARG;
+    ANPD_TRY(check_device(m));
     if (kv->h_kv_len[seq] != 0) return ANPD_ERR_STATE;
     if (prompt_len + ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
     for (int i = 0; i < prompt_len; ++i) if (prompt[i] < 0 || prompt[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
@@ -525,6 +535,7 @@ anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_to
 // the batch * 8 rows, argmax / accept and, in COMMIT mode, the KV commit and token-buffer append.
 // Steps of one shape are captured once into a CUDA graph and replayed.
 static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K = -1) {
+    ANPD_TRY(check_device(m));
     int max_pos = 0;
     for (int b = 0; b < kv->batch; ++b) {
         // the attention grid is sized from the host's copy of the lengths: it must not be behind the device
@@ -543,10 +554,8 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
     };
     if (m->prof.on || !kv->use_graphs || !kv->warm) {
         kv->warm = true;
-        const bool pdl = g_use_pdl;
-        if (m->prof.on) g_use_pdl = false;            // per-launch timing needs kernels that do not overlap
+        NoPdlScope no_overlap(m->prof.on);            // per-launch timing needs kernels that do not overlap
         const anpd_status rc = enqueue();
-        g_use_pdl = pdl;
         if (rc == ANPD_OK && mode == ACCEPT_COMMIT) std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1);
         return rc;
     }
@@ -554,7 +563,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
                          ((uint64_t)(want_logits ? 1 : 0) << 28) | ((uint64_t)(d_ctxs ? 1 : 0) << 29);
     auto it = kv->graphs.find(key);
     if (it == kv->graphs.end()) {
-        const long long before = g_launch_count;
+        const long long before = g_launch_count.load();
         cudaGraph_t graph = nullptr;
         if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
             cudaGetLastError();
@@ -563,8 +572,8 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
         }
         const anpd_status rc = enqueue();
         const cudaError_t ce = cudaStreamEndCapture(st, &graph);
-        const int launches = (int)(g_launch_count - before);
-        g_launch_count = before;                      // capturing runs nothing
+        const int launches = (int)(g_launch_count.load() - before);
+        g_launch_count.fetch_sub(launches);           // capturing runs nothing
         anpd_kv::StepGraph sg{nullptr, launches};
         if (rc != ANPD_OK || ce != cudaSuccess || !graph || cudaGraphInstantiate(&sg.exec, graph, 0) != cudaSuccess) {
             cudaGetLastError();
@@ -635,6 +644,7 @@ static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* 
                                  int prompt_len, int max_new, int K, int32_t* out, anpd_stats* stats, bool on_device) {
     if (!m || !kv || kv->m != m || !ctxs || !prompts || !out || prompt_len < 1 || max_new < 1) return ANPD_ERR_ARG;
     if (K < 0 || K > ANPD_K_MAX) return ANPD_ERR_RANGE;
+    ANPD_TRY(check_device(m));
     const int B = kv->batch;
     cudaStream_t st = m->stream;
     for (int b = 0; b < B; ++b) {

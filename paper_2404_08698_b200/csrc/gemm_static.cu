@@ -126,7 +126,13 @@ extern "C" anpd_status anpd_gemm_static(const uint16_t* w_bf16_dev, int N, int K
     CUtensorMap mh, ml;
     ANPD_TRY(make_tmap_bf16(&mh, d_hi, rows, K, NB, false));
     ANPD_TRY(make_tmap_bf16(&ml, d_lo, rows, K, NB, false));
-    ANPD_TRY(gemm_tc_enqueue(plan, d_w, mh, ml, rows, NB, d_part, (size_t)rows * N, N, d_err, st, nullptr));
+    {
+        // The GEMM kernel requests its first weight blocks ahead of its dependency wait, which is only sound for
+        // weights no earlier kernel of the stream writes.  Here the blocks were written by the kernels just above,
+        // so this launch must not overlap them: no programmatic dependent launch.
+        NoPdlScope ordered(true);
+        ANPD_TRY(gemm_tc_enqueue(plan, d_w, mh, ml, rows, NB, d_part, (size_t)rows * N, N, d_err, st, nullptr));
+    }
     static_reduce_kernel<<<64, 256, 0, st>>>(d_part, plan.d_seg_count, rows, N, out_dev);
     CUDA_TRY(cudaGetLastError());
     int err = 0;

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <atomic>
 #include <map>
 #include <vector>
 
@@ -61,7 +62,7 @@ struct Profiler {
     ~Profiler();
 };
 
-extern long long g_launch_count;
+extern std::atomic<long long> g_launch_count;
 
 // Wraps one kernel launch: counts it and, when profiling, brackets it with events.
 #define LAUNCH(prof, stream, kclass, wbytes, ...)                      \
@@ -81,8 +82,17 @@ extern long long g_launch_count;
 // The weight-streaming GEMM uses the gap: its producer thread requests the first weight tiles before
 // it waits, so HBM keeps streaming through the small kernels between two GEMMs.  A kernel launched
 // without the attribute (or with ANPD_NO_PDL set) sees both calls as no-ops.
+// g_use_pdl is fixed when the library is loaded; t_no_pdl switches the attribute off for the launches
+// the calling thread makes while it is set (per-launch timing; a GEMM whose weights were written by
+// the kernel just before it and must therefore not be requested ahead of the dependency wait).
 // ---------------------------------------------------------------------------------------------
-extern bool g_use_pdl;
+extern const bool g_use_pdl;
+extern thread_local bool t_no_pdl;
+struct NoPdlScope {
+    bool saved;
+    explicit NoPdlScope(bool off) : saved(t_no_pdl) { if (off) t_no_pdl = true; }
+    ~NoPdlScope() { t_no_pdl = saved; }
+};
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -95,7 +105,7 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_use_pdl ? 1 : 0;
+    cfg.numAttrs = (g_use_pdl && !t_no_pdl) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 #endif
@@ -206,6 +216,7 @@ struct anpd_model {
     int max_segs;
     bool plain_gemm;                  // debugging aid: route GEMMs through the plain kernel
     int num_sms;
+    int device;                       // ordinal of the device the weight blocks were laid out for
     Profiler prof;
 };
 

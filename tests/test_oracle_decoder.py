@@ -199,3 +199,14 @@ def test_bf16_cache_incremental_equals_full():
     a = dec16.forward(toks[:4], c)
     b = dec16.forward(toks[4:], c)
     assert torch.allclose(torch.cat([a, b]), full, atol=1e-12, rtol=0)
+
+
+def test_keep_cast_changes_no_value():
+    # casting each weight once and keeping the copy is the same arithmetic on the same values
+    w = make_weights(SMALL, 5, True, std=0.3)                       # bf16 matrices: a real cast happens
+    toks = [3, 9, 27, 5, 1]
+    for dtype in (torch.float32, torch.float64):
+        a, b = Decoder(SMALL, w, dtype), Decoder(SMALL, w, dtype, keep_cast=True)
+        ca, cb = a.new_cache(), b.new_cache()
+        for chunk in (toks[:3], toks[3:]):                          # second call uses the kept copies
+            assert torch.equal(a.forward(chunk, ca), b.forward(chunk, cb))
