@@ -1,0 +1,129 @@
+"""Logit parity at the REAL widths and at the context lengths the benchmark runs, against the PLAIN fp64 oracle at
+the stated bar of 2e-2 max-abs.
+
+A model of the full depth cannot be compared with the plain oracle at that bar (through 22-40 random layers the
+bf16 rounding of the cache alone moves the oracle's own logits by more than it; tests/test_gpu_fullsize.py covers
+the full depth against the oracle with the bf16 cache).  One layer does not amplify the cache's rounding, and it
+still runs every kernel in its full-size configuration: the stream-K GEMM plans of the real matrix shapes over
+all SMs, the paged attention over 17 / 33 key pages per head (both slot configurations of the tensor-memory
+kernel), eight query heads per kv head at head dimension 64, and the LM head over 32000 tokens.
+
+The second half runs the 1.1B and the 7B workloads at full length and compares the produced stream with ONE
+teacher-forced oracle forward over prompt + stream (bf16-cache oracle, since the cache precision is part of the
+workload): the stream's token must be the oracle's argmax wherever the oracle's top-2 margin exceeds the bar.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import gpu_model, new_stream, require_gpu
+from oracle.decoder import Decoder
+from workloads import WORKLOADS, ModelShape, make_prompts, make_weights, markov_prompt
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = 2e-2      # max-abs, bf16 GPU against the plain oracle
+MARGIN = 5e-2         # decisions are compared where the oracle's top-2 margin exceeds this
+
+
+@pytest.fixture(scope="module")
+def A():
+    require_gpu()
+    from paper_2404_08698_b200 import binding
+    return binding
+
+
+ONE_LAYER_CASES = [
+    # shape (one layer of ...),                                    prompt length, what it exercises
+    (ModelShape(1, 4096, 32, 32, 128, 11008, 32000), 2048),        # 7B width, 17 pages: four attention slots per SM
+    (ModelShape(1, 4096, 32, 32, 128, 11008, 32000), 4096),        # 7B width, 33 pages: five slots, two items per slot
+    (ModelShape(1, 5120, 40, 40, 128, 13824, 32000), 2048),        # 13B width: other GEMM splits
+    (ModelShape(1, 2048, 32, 4, 64, 5632, 32000), 768),            # 1.1B width: 8 query heads per kv head, hd 64
+]
+
+
+@pytest.mark.parametrize("shape,plen", ONE_LAYER_CASES, ids=lambda v: str(v) if isinstance(v, int) else f"d{v.d_model}")
+def test_one_layer_at_real_width_against_plain_oracle(A, shape, plen):
+    w = make_weights(shape, 11, True, device="cuda")
+    torch.cuda.synchronize()
+    m = gpu_model(A, shape, w, new_stream())
+    w_cpu = {k: v.cpu() for k, v in w.items()}
+    del w
+    torch.cuda.empty_cache()
+    prompt = markov_prompt(plen, shape.vocab, 3, 4242 + plen, copy_spans=True).tolist()
+    draft = [int(t) for t in markov_prompt(7, shape.vocab, 3, 99)]
+    kv = A.anpd_kv_create(m, plen + 64)
+    try:
+        first = A.anpd_prefill(m, kv, prompt)
+        got = A.anpd_verify_logits(m, kv, first, draft, shape.vocab)          # all 8 rows
+    finally:
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(m)
+    dec = Decoder(shape, w_cpu, torch.float64)                                # the plain definition: full-precision cache
+    cache = dec.new_cache()
+    lp = dec.forward(prompt, cache)
+    want = dec.forward([first] + draft, cache)
+    t2 = torch.topk(lp[-1], 2).values
+    if float(t2[0] - t2[1]) > MARGIN:
+        assert first == int(torch.argmax(lp[-1]))
+    diff = (torch.from_numpy(got).double() - want).abs()
+    sigma = float(want.std())
+    err = float(diff.max())
+    print(f"d{shape.d_model} hd{shape.head_dim} ctx {plen}: max-abs {err:.2e}, rms {float(diff.pow(2).mean().sqrt()):.2e}, "
+          f"logit sigma {sigma:.3f}, max-abs / sigma {err / sigma:.2e}")
+    assert err <= LOGIT_TOL, err
+    for r in range(want.shape[0]):
+        t2 = torch.topk(want[r], 2).values
+        if float(t2[0] - t2[1]) > MARGIN:
+            assert int(np.argmax(got[r])) == int(torch.argmax(want[r])), r
+
+
+def _full_length_stream_check(A, wl, dtype, margin):
+    """Greedy and ANPD streams of the workload at full length; returns (decided, total, worst margin of a
+    disagreement) of the teacher-forced comparison with the bf16-cache oracle."""
+    w = make_weights(wl.shape, wl.weight_seed, True, device="cuda")
+    torch.cuda.synchronize()
+    st = new_stream()
+    m = gpu_model(A, wl.shape, w, st)
+    w_cpu = {k: v.cpu() for k, v in w.items()}
+    del w
+    torch.cuda.empty_cache()
+    prompt = make_prompts(wl)[0]
+    max_len = wl.prompt_len + wl.max_new + 64
+    kv = A.anpd_kv_create(m, max_len)
+    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, st)
+    try:
+        greedy, _ = A.anpd_generate(m, kv, ctx, prompt, wl.max_new, 0)
+        out, _ = A.anpd_generate(m, kv, ctx, prompt, wl.max_new, wl.K)
+    finally:
+        A.anpd_ngram_destroy(ctx)
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(m)
+    assert np.array_equal(out, greedy)
+    # one causal forward over prompt + stream[:-1] gives, at position len(prompt)-1+i, the logits that decide stream[i]
+    dec = Decoder(wl.shape, w_cpu, dtype, kv_dtype=torch.bfloat16)
+    seq = prompt.tolist() + greedy.tolist()[:-1]
+    logits = dec.forward(seq, dec.new_cache())[len(prompt) - 1:]
+    top = torch.topk(logits, 2, dim=-1)
+    margins = (top.values[:, 0] - top.values[:, 1]).double()
+    agree = top.indices[:, 0] == torch.from_numpy(greedy.astype(np.int64))
+    worst = float(margins[~agree].max()) if bool((~agree).any()) else 0.0
+    decided = int((margins > margin).sum())
+    return decided, len(greedy), worst, int((~agree).sum())
+
+
+def test_c2_full_length_stream_against_teacher_forced_oracle(A):
+    """1.1B workload, prompt 512 + 256 generated tokens, fp64 oracle with the bf16 cache."""
+    decided, total, worst, n_diff = _full_length_stream_check(A, WORKLOADS["C2"], torch.float64, MARGIN)
+    print(f"C2: {decided}/{total} tokens decided above {MARGIN}; {n_diff} disagreements, the largest at margin {worst:.3e}")
+    assert worst <= MARGIN, worst              # every disagreement lies under the margin
+    assert decided >= total // 4, decided
+
+
+def test_c3_full_length_stream_against_teacher_forced_oracle(A):
+    """7B workload, prompt 1536 + 256 generated tokens.  The oracle runs in its fp32 mode here (1792 tokens through
+    6.6 G parameters; fp32 rounding, about 1e-6 relative, is far below the margin) with the bf16 cache."""
+    decided, total, worst, n_diff = _full_length_stream_check(A, WORKLOADS["C3"], torch.float32, MARGIN)
+    print(f"C3: {decided}/{total} tokens decided above {MARGIN}; {n_diff} disagreements, the largest at margin {worst:.3e}")
+    assert worst <= MARGIN, worst
+    assert decided >= total // 4, decided

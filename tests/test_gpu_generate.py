@@ -5,8 +5,8 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import as_bf16_values, check_stream_against_oracle, gpu_model, new_stream, require_gpu
-from oracle.anpd import anpd_generate as oracle_anpd
+from helpers import as_bf16_values, check_stream_against_oracle, gpu_model, new_stream, require_gpu, top2_margin
+from oracle.anpd import argmax_lowest, verify as oracle_verify
 from oracle.decoder import Decoder
 from oracle.mln import MLN
 from workloads import WORKLOADS, ModelShape, make_prompts, make_weights, markov_prompt, periodic_prompt
@@ -49,12 +49,69 @@ def test_c1_anpd_equals_greedy_equals_oracle(A, c1):
         dec = Decoder(wl.shape, as_bf16_values(w), torch.float64)
         n = check_stream_against_oracle(dec, prompt.tolist(), ref.tolist())
         assert n >= wl.max_new // 5, n
-        # the oracle's Algorithm 1 on the same stream: if its own greedy stream is the library's,
-        # it must have taken the same steps (same drafts, same accepted lengths)
-        want, ost, _ = oracle_anpd(dec, prompt.tolist(), wl.max_new, wl.K, n_max=wl.n_max)
-        if want == ref.tolist():
-            assert st["steps"] == ost.steps and st["accepted"] == ost.accepted and st["drafted"] == ost.drafted
-            assert st["hist_accepted"] == ost.hist_accepted
+    finally:
+        A.anpd_ngram_destroy(ctx)
+
+
+def test_algorithm1_step_by_step_from_the_boundary_calls(A, c1):
+    """Algorithm 1 driven from the host through anpd_ngram_update -> anpd_ngram_draft -> anpd_verify, compared
+    with the oracle at EVERY step: the draft bit for bit, the accepted length and the next token wherever every
+    logit row that decides them has a top-2 margin above 5e-2 in the oracle.  Where a decision falls under the
+    margin and the two sides differ, the oracle is put on the library's path (its cache rolled back or extended
+    to the library's accepted length), so that all later steps are compared too."""
+    wl, w, m, kv, st = c1
+    prompt = make_prompts(wl)[0].tolist()
+    K, M, MARGIN = wl.K, wl.max_new, 5e-2
+    dec = Decoder(wl.shape, as_bf16_values(w), torch.float64)
+    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, 512, 0, st)
+    try:
+        A.anpd_kv_truncate(kv, 0, 0)
+        mln = MLN(wl.n_min, wl.n_max)
+        mln.initialize(prompt)
+        A.anpd_ngram_update(ctx, prompt)
+        cache = dec.new_cache()
+        logits = dec.forward(prompt, cache)
+        confirmed = A.anpd_prefill(m, kv, prompt)
+        if top2_margin(logits[-1]) > MARGIN:
+            assert confirmed == argmax_lowest(logits[-1])
+        out, steps, decided, accepted_total = [], 0, 0, 0
+        while len(out) < M:
+            out.append(confirmed)
+            mln.update(confirmed)
+            A.anpd_ngram_update(ctx, [confirmed])
+            want_draft = mln.draft(K)
+            draft = A.anpd_ngram_draft(ctx, K)
+            assert draft == want_draft, (steps, draft, want_draft)                  # bit-exact, every step
+            P = cache.length
+            a_o, nxt_o, preds, lg = oracle_verify(dec, cache, confirmed, draft)
+            a, nxt = A.anpd_verify(m, kv, confirmed, draft)
+            assert A.anpd_kv_len(kv) == P + a + 1
+            # rows 0..min(a, a_o) decide the accepted length; row a decides the next token
+            rows = range(min(a, a_o) + 1)
+            clear = all(top2_margin(lg[r]) > MARGIN for r in rows)
+            if clear:
+                assert a == a_o and nxt == nxt_o, (steps, a, a_o, nxt, nxt_o)
+                decided += 1
+            if a != a_o:                                                           # only possible under the margin
+                if a > a_o:
+                    dec.forward(draft[a_o:a], cache)
+                else:
+                    cache.truncate(P + a + 1)
+            assert cache.length == P + a + 1
+            for t in draft[:a]:
+                out.append(t)
+                mln.update(t)
+            if a:
+                A.anpd_ngram_update(ctx, draft[:a])
+            accepted_total += a
+            confirmed = nxt
+            steps += 1
+        assert decided >= steps // 2 and decided >= 8, (decided, steps)
+        assert accepted_total > 0
+        # the library's own loop takes the same steps
+        got, gst = A.anpd_generate(m, kv, ctx, prompt, M, K)
+        assert got.tolist() == out[:M]
+        assert gst["steps"] == steps and gst["accepted"] == accepted_total
     finally:
         A.anpd_ngram_destroy(ctx)
 

@@ -47,6 +47,15 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point(A):
     assert np.array_equal(got1, want1) and np.array_equal(got2, want2)
 
 
+def test_same_shape_other_weights_uses_the_new_weights(A):
+    """Two calls of one shape with different weights: the second must see its own weight blocks in the
+    shared scratch, not the first call's (the GEMM may not fetch them ahead of the kernel that writes them)."""
+    got1, want1 = one_call(A, 640, 448, 8, seed=51)
+    got2, want2 = one_call(A, 640, 448, 8, seed=52)
+    assert np.array_equal(got1, want1) and np.array_equal(got2, want2)
+    assert not np.array_equal(got1, got2)
+
+
 def test_sizes_beyond_the_fixed_scratch_are_rejected(A):
     w = torch.zeros(4096, 4096, dtype=torch.bfloat16, device="cuda")   # 32 x 64 = 2048 blocks > 128
     a = torch.zeros(8, 4096, device="cuda")
