@@ -236,8 +236,10 @@ long long anpd_launch_count(int reset);
 /* Test hook for the projections inside LLM(drafts) (Section 3.1, "Verification"):
  * out[rows][N] = A[rows][K] x W[N][K]^T through the library's weight-streaming GEMM kernel, on
  * the current device and the default stream.  W: N*K bf16 bit patterns (host); A: rows*K fp32
- * (host), rows a multiple of 8 and at most 128; K a multiple of 8.  plain != 0 selects the
- * reference kernel the tensor-core kernel is cross-checked against. */
+ * (host), rows a multiple of 8 and at most 128; K a multiple of 8.  plain: 0 = the stream-K
+ * tensor-core kernel (steps of several sequences, prefill passes), 1 = the one-warp-per-feature
+ * kernel it is cross-checked against, 2 = the row-range tensor-core kernel of single-sequence
+ * steps (rows must be 8). */
 anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a, int rows, float* out, int plain);
 
 /* The same product as anpd_debug_gemm for callers that must not allocate device memory; the paper

@@ -333,8 +333,9 @@ def anpd_launch_count(reset: bool = False) -> int:
     return int(lib().anpd_launch_count(int(reset)))
 
 
-def anpd_debug_gemm(w_bf16, a, plain: bool = False) -> np.ndarray:
-    """w_bf16: torch bf16 CPU tensor [N, K]; a: fp32 array [rows, K].  Returns out [rows, N] fp32."""
+def anpd_debug_gemm(w_bf16, a, plain: int = 0) -> np.ndarray:
+    """w_bf16: torch bf16 CPU tensor [N, K]; a: fp32 array [rows, K].  Returns out [rows, N] fp32.
+    plain: 0 stream-K kernel, 1 plain cross-check kernel, 2 row-range kernel (8 rows)."""
     import torch
     N, K = w_bf16.shape
     wb = np.ascontiguousarray(w_bf16.contiguous().view(torch.int16).numpy().view(np.uint16))

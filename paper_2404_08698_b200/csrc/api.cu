@@ -208,13 +208,26 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
         const int shapes[GK_COUNT][2] = {{m->nqkv, c.d_model}, {c.d_model, m->dq}, {2 * c.d_ffn, c.d_model}, {c.d_model, c.d_ffn},
                                          {c.vocab, c.d_model}};
         for (int k = 0; k < GK_COUNT; ++k) gemm_make_plan(&m->plan[k], shapes[k][0], shapes[k][1], sms);
+        for (int k = 0; k < GK_COUNT; ++k) rr_make_plan(&m->rr[k], shapes[k][0], shapes[k][1], sms);
     }
+    m->rr_slab = nullptr;
+    m->rr_lm = nullptr;
+    // single-sequence steps run on a second copy of the projections in row-range storage (ANPD_NO_RR=1: stream-K only)
+    m->rr_ready = std::getenv("ANPD_NO_RR") == nullptr;
+    for (int k = 0; k < GK_COUNT; ++k)
+        if (m->rr[k].mt > 2) m->rr_ready = false;      // a CTA's feature range must fit two 128-row MMA tiles (very large vocabularies do not)
     const size_t b_embed = up256(V * d * 2), b_lm = up256(gemm_tiled_elems(m->plan[GK_LM]) * 2),
                  b_qkv = up256(gemm_tiled_elems(m->plan[GK_QKV]) * 2), b_o = up256(gemm_tiled_elems(m->plan[GK_O]) * 2),
                  b_gu = up256(gemm_tiled_elems(m->plan[GK_GU]) * 2), b_d = up256(gemm_tiled_elems(m->plan[GK_DOWN]) * 2),
                  b_norm = up256(d * 4);
     m->slab_bytes = b_embed + b_lm + b_norm + c.n_layers * (b_qkv + b_o + b_gu + b_d + 2 * b_norm);
     if (cudaMalloc(&m->slab, m->slab_bytes) != cudaSuccess) { cudaGetLastError(); delete m; return ANPD_ERR_OOM; }
+    size_t rr_bytes[GK_COUNT], rr_total = 0;
+    for (int k = 0; k < GK_COUNT; ++k) {
+        rr_bytes[k] = up256(rr_storage_bytes(m->rr[k]));
+        rr_total += rr_bytes[k] * (k == GK_LM ? 1 : (size_t)c.n_layers);
+    }
+    if (m->rr_ready && cudaMalloc(&m->rr_slab, rr_total) != cudaSuccess) { cudaGetLastError(); cudaFree(m->slab); delete m; return ANPD_ERR_OOM; }
     m->streamed_bytes = 2.0 * ((double)c.n_layers * ((double)m->nqkv * d + (double)d * m->dq + 3.0 * F * d) + (double)V * d);
 
     char* p = (char*)m->slab;
@@ -225,16 +238,18 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     // staging for host-side sources: the largest matrix in its source type
     void* stage = nullptr;
     const size_t max_elems = std::max(std::max((size_t)V * d, F * d), std::max((size_t)m->dq * d, d * F));
-    if (!dev && cudaMalloc(&stage, max_elems * (bf ? 2 : 4)) != cudaSuccess) { cudaGetLastError(); cudaFree(m->slab); delete m; return ANPD_ERR_OOM; }
+    if (!dev && cudaMalloc(&stage, max_elems * (bf ? 2 : 4)) != cudaSuccess) { cudaGetLastError(); cudaFree(m->rr_slab); cudaFree(m->slab); delete m; return ANPD_ERR_OOM; }
     if (cudaMemsetAsync(m->slab, 0, m->slab_bytes, st) != cudaSuccess) rc = ANPD_ERR_CUDA;
+    if (m->rr_ready && cudaMemsetAsync(m->rr_slab, 0, rr_total, st) != cudaSuccess) rc = ANPD_ERR_CUDA;
+    unsigned char* rp = (unsigned char*)m->rr_slab;     // next free byte of the row-range storage
     auto put = [&](const void* src, size_t n, bool as_bf16, size_t bytes) -> void* {
         void* dst = p;
         p += bytes;
         if (rc == ANPD_OK) rc = upload(dst, src, n, as_bf16, bf, dev, st, tmp, nullptr, 0);
         return dst;
     };
-    // rows [row_off, row_off + rows) of a tiled [*, K] matrix at dst
-    auto put_tiled = [&](int kind, const void* src, int rows, int K, int row_off, void* dst) {
+    // rows [row_off, row_off + rows) of a tiled [*, K] matrix at dst, and of its row-range copy at rdst
+    auto put_tiled = [&](int kind, const void* src, int rows, int K, int row_off, void* dst, unsigned char* rdst) {
         if (rc != ANPD_OK) return;
         const void* dsrc = src;
         if (!dev) {
@@ -243,41 +258,52 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
             dsrc = stage;
         }
         rc = gemm_retile_enqueue(m->plan[kind], dsrc, !bf, rows, row_off, (bf16*)dst, st);
+        if (rc == ANPD_OK && m->rr_ready) {
+            const int map = kind == GK_QKV ? RR_MAP_HEADS : kind == GK_GU ? RR_MAP_GATE_UP : RR_MAP_IDENTITY;
+            rc = rr_retile_enqueue(m->rr[kind], dsrc, !bf, rows, row_off, map, c.head_dim, c.d_ffn, rdst, st);
+        }
         if (rc == ANPD_OK && !dev && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
     };
     int t = 0;
     m->embed = (const bf16*)put(weights[t++], V * d, true, b_embed);
     m->layers.resize(c.n_layers);
+    m->rr_layers.resize(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l) {
         LayerW& w = m->layers[l];
+        anpd_model::LayerRR& r = m->rr_layers[l];
         w.attn_norm = (const float*)put(weights[t++], d, false, b_norm);
         // q, k and v rows form one matrix so that one GEMM produces all three
         w.wqkv = (const bf16*)p;
-        put_tiled(GK_QKV, weights[t++], m->dq, (int)d, 0, p);
-        put_tiled(GK_QKV, weights[t++], m->dkv, (int)d, m->dq, p);
-        put_tiled(GK_QKV, weights[t++], m->dkv, (int)d, m->dq + m->dkv, p);
-        p += b_qkv;
+        r.wqkv = rp;
+        put_tiled(GK_QKV, weights[t++], m->dq, (int)d, 0, p, rp);
+        put_tiled(GK_QKV, weights[t++], m->dkv, (int)d, m->dq, p, rp);
+        put_tiled(GK_QKV, weights[t++], m->dkv, (int)d, m->dq + m->dkv, p, rp);
+        p += b_qkv; rp += rr_bytes[GK_QKV];
         w.wo = (const bf16*)p;
-        put_tiled(GK_O, weights[t++], (int)d, m->dq, 0, p);
-        p += b_o;
+        r.wo = rp;
+        put_tiled(GK_O, weights[t++], (int)d, m->dq, 0, p, rp);
+        p += b_o; rp += rr_bytes[GK_O];
         w.ffn_norm = (const float*)put(weights[t++], d, false, b_norm);
         w.wgu = (const bf16*)p;
-        put_tiled(GK_GU, weights[t++], (int)F, (int)d, 0, p);
-        put_tiled(GK_GU, weights[t++], (int)F, (int)d, (int)F, p);
-        p += b_gu;
+        r.wgu = rp;
+        put_tiled(GK_GU, weights[t++], (int)F, (int)d, 0, p, rp);
+        put_tiled(GK_GU, weights[t++], (int)F, (int)d, (int)F, p, rp);
+        p += b_gu; rp += rr_bytes[GK_GU];
         w.wd = (const bf16*)p;
-        put_tiled(GK_DOWN, weights[t++], (int)d, (int)F, 0, p);
-        p += b_d;
+        r.wd = rp;
+        put_tiled(GK_DOWN, weights[t++], (int)d, (int)F, 0, p, rp);
+        p += b_d; rp += rr_bytes[GK_DOWN];
     }
     m->final_norm = (const float*)put(weights[t++], d, false, b_norm);
     m->lm_head = (const bf16*)p;
-    put_tiled(GK_LM, weights[t++], (int)V, (int)d, 0, p);
+    m->rr_lm = rp;
+    put_tiled(GK_LM, weights[t++], (int)V, (int)d, 0, p, rp);
     p += b_lm;
     if (rc == ANPD_OK && cudaStreamSynchronize(st) != cudaSuccess) { anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__); rc = ANPD_ERR_CUDA; }
     if (stage) cudaFree(stage);
     m->d_plan_tables = nullptr;
     if (rc == ANPD_OK) rc = model_make_plans(m);
-    if (rc != ANPD_OK) { cudaFree(m->d_plan_tables); cudaFree(m->slab); delete m; return rc; }
+    if (rc != ANPD_OK) { cudaFree(m->d_plan_tables); cudaFree(m->rr_slab); cudaFree(m->slab); delete m; return rc; }
     *out = m;
     return ANPD_OK;
 }
@@ -286,6 +312,7 @@ anpd_status anpd_model_destroy(anpd_model* m) {
     if (!m) return ANPD_ERR_ARG;
     cudaStreamSynchronize(m->stream);
     cudaFree(m->d_plan_tables);
+    cudaFree(m->rr_slab);
     cudaFree(m->slab);
     delete m;
     return ANPD_OK;
@@ -335,7 +362,13 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&ws.logits, R * V * 4},
         {(void**)&ws.amax_val, R * ws.amax_blocks * 4}, {(void**)&ws.amax_idx, R * ws.amax_blocks * 4},
         {(void**)&ws.gemm_err, 256},
+        {(void**)&ws.img_h, act_img_bytes(c.d_model)}, {(void**)&ws.img_h2, act_img_bytes(c.d_model)},
+        {(void**)&ws.img_ao, act_img_bytes(m->dq)}, {(void**)&ws.img_act, act_img_bytes(c.d_ffn)},
+        {(void**)&ws.ss_a, (size_t)m->num_sms * ANPD_ROWS * 4}, {(void**)&ws.ss_b, (size_t)m->num_sms * ANPD_ROWS * 4},
+        {(void**)&ws.amax_val_rr, (size_t)m->num_sms * ANPD_ROWS * 4}, {(void**)&ws.amax_idx_rr, (size_t)m->num_sms * ANPD_ROWS * 4},
     };
+    ws.amax_nblk = ws.amax_blocks;
+    ws.amax_rr = false;
     size_t total = 0;
     for (const Item& it : items) total += up256(it.bytes);
     kv->slab_bytes = total;
@@ -755,9 +788,51 @@ anpd_status anpd_generate_dev(anpd_model* m, anpd_kv* kv, anpd_ngram* ctx, const
 // ---------------------------------------------------------------------------------------------
 // GEMM test hook
 // ---------------------------------------------------------------------------------------------
+// The product through the row-range kernel of single-sequence steps (exactly 8 rows), plain epilogue.
+static anpd_status debug_gemm_row_range(const uint16_t* w_bf16, int N, int K, const float* a, float* out) {
+    int dev = 0, sms = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    RRPlan plan;
+    rr_make_plan(&plan, N, K, sms);
+    const size_t wb = up256(rr_storage_bytes(plan)), ib = up256(act_img_bytes(K)), sb = up256((size_t)N * K * 2),
+                 ab = up256((size_t)ANPD_ROWS * K * 4), ob = up256((size_t)ANPD_ROWS * N * 4);
+    char* slab = nullptr;
+    if (cudaMalloc((void**)&slab, wb + ib + sb + ab + ob + 256) != cudaSuccess) { cudaGetLastError(); return ANPD_ERR_OOM; }
+    unsigned char* dW = (unsigned char*)slab;
+    unsigned char* dimg = dW + wb;
+    void* dsrc = dimg + ib;
+    float* da = (float*)((char*)dsrc + sb);
+    float* dout = (float*)((char*)da + ab);
+    int* derr = (int*)((char*)dout + ob);
+    auto body = [&]() -> anpd_status {
+        CUDA_TRY(cudaMemset(slab, 0, wb + ib));
+        CUDA_TRY(cudaMemset(dout, 0, ob + 256));
+        CUDA_TRY(cudaMemcpy(dsrc, w_bf16, (size_t)N * K * 2, cudaMemcpyHostToDevice));
+        CUDA_TRY(cudaMemcpy(da, a, (size_t)ANPD_ROWS * K * 4, cudaMemcpyHostToDevice));
+        ANPD_TRY(rr_retile_enqueue(plan, dsrc, false, N, 0, RR_MAP_IDENTITY, 0, 0, dW, 0));
+        ANPD_TRY(rr_act_image_enqueue(da, K, dimg, 0));
+        CUDA_TRY(cudaDeviceSynchronize());
+        RREpiHost e;
+        e.raw_out = dout;
+        ANPD_TRY(rr_enqueue(RR_RAW, plan, dW, dimg, e, derr, 0, nullptr));
+        CUDA_TRY(cudaDeviceSynchronize());
+        int err = 0;
+        CUDA_TRY(cudaMemcpy(&err, derr, 4, cudaMemcpyDeviceToHost));
+        if (err) { std::snprintf(g_last_error, sizeof(g_last_error), "GEMM kernel gave up waiting (code %d)", err); return ANPD_ERR_CUDA; }
+        CUDA_TRY(cudaMemcpy(out, dout, (size_t)ANPD_ROWS * N * 4, cudaMemcpyDeviceToHost));
+        return ANPD_OK;
+    };
+    const anpd_status rc = body();
+    cudaFree(slab);
+    return rc;
+}
+
 anpd_status anpd_debug_gemm(const uint16_t* w_bf16, int N, int K, const float* a, int rows, float* out, int plain) {
     if (!w_bf16 || !a || !out || N < 1 || K < 8 || K % 8 || rows < 8 || rows % 8 || rows > 128) return ANPD_ERR_ARG;
+    if (plain == 2 && rows != ANPD_ROWS) return ANPD_ERR_ARG;
     if (!have_device()) return ANPD_ERR_CUDA;
+    if (plain == 2) return debug_gemm_row_range(w_bf16, N, K, a, out);
     int dev = 0, sms = 0;
     CUDA_TRY(cudaGetDevice(&dev));
     CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));

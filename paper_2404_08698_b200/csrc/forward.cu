@@ -119,6 +119,34 @@ __global__ void __launch_bounds__(NORM_THREADS) embed_norm_kernel(const bf16* __
     }
 }
 
+// Single-sequence steps (row-range projections): x = E[tok]; the first projection's operand image receives
+// x * gain as hi + lo terms, un-normalised; the row's sum of squares goes to ss[0][row] (one partial).
+__global__ void __launch_bounds__(NORM_THREADS) embed_img_kernel(const bf16* __restrict__ embed, const int* __restrict__ row_tok,
+                                                                 const float* __restrict__ gain, int d, float* __restrict__ x,
+                                                                 unsigned char* __restrict__ img, float* __restrict__ ss) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float red[32];
+    const int row = blockIdx.x, chunks = d >> 2;
+    const bf16* e = embed + (size_t)row_tok[row] * d;
+    float acc = 0.0f;
+    for (int c = threadIdx.x; c < chunks; c += NORM_THREADS) {
+        const uint2 raw = *(const uint2*)(e + 4 * c);
+        const bf16* b = (const bf16*)&raw;
+        const float4 g = *(const float4*)(gain + 4 * c);
+        const float v[4] = {__bfloat162float(b[0]), __bfloat162float(b[1]), __bfloat162float(b[2]), __bfloat162float(b[3])};
+        const float gg[4] = {g.x, g.y, g.z, g.w};
+        *(float4*)(x + (size_t)row * d + 4 * c) = make_float4(v[0], v[1], v[2], v[3]);
+        bf16 hi[4], lo[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { split_bf16(v[t] * gg[t], hi[t], lo[t]); acc += v[t] * v[t]; }
+        *(uint2*)(img + act_img_offset(row, 4 * c)) = *(const uint2*)hi;               // 4 elements never straddle a 16-byte chunk
+        *(uint2*)(img + act_img_offset(ANPD_ROWS + row, 4 * c)) = *(const uint2*)lo;
+    }
+    const float t = block_sum_1024(acc, red);
+    if (threadIdx.x == 0) ss[row] = t;
+}
+
 // x[row] += sum of the tile's partial sums (in segment order); then h = rmsnorm(x) * gain as hi + lo.
 __global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part,
                                                                   const int* __restrict__ seg_count, size_t split_stride, int ld_part,
@@ -456,7 +484,7 @@ constexpr int COMBINE_SLICES = 4;
 constexpr int COMBINE_MAX_PAGES = 256;
 __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* __restrict__ pl, const float* __restrict__ po,
                                     const int* __restrict__ row_pos, int Hq, int hd, int pages_per_seq,
-                                    bf16* __restrict__ ao_hi, bf16* __restrict__ ao_lo) {
+                                    bf16* __restrict__ ao_hi, bf16* __restrict__ ao_lo, unsigned char* __restrict__ img) {
     pdl_trigger();
     pdl_wait();
     __shared__ float s_w[COMBINE_MAX_PAGES];            // page maxima, then page weights
@@ -500,9 +528,14 @@ __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* _
         for (int k = 1; k < COMBINE_SLICES; ++k) t += s_o[k][dim];
         bf16 hi, lo;
         split_bf16(t / s_L, hi, lo);
-        const size_t out = (size_t)row * Hq * hd + head * hd + dim;
-        ao_hi[out] = hi;
-        ao_lo[out] = lo;
+        if (img) {                                        // single-sequence step: straight into the O projection's operand image
+            *(bf16*)(img + act_img_offset(row, head * hd + dim)) = hi;
+            *(bf16*)(img + act_img_offset(ANPD_ROWS + row, head * hd + dim)) = lo;
+        } else {
+            const size_t out = (size_t)row * Hq * hd + head * hd + dim;
+            ao_hi[out] = hi;
+            ao_lo[out] = lo;
+        }
     }
 }
 
@@ -773,7 +806,7 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
 }
 
 template <int HD>
-anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos) {
+anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, unsigned char* img = nullptr) {
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * HD;
@@ -798,7 +831,7 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
                      ws.row_pos, c.n_q_heads, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
     else LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
-                                                                              HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
+                                                                              HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo, img)));
     return ANPD_OK;
 }
 
@@ -835,15 +868,64 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
 anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len) {
     Workspace& ws = kv->ws;
     const int blocks = (mode == ACCEPT_PREFILL) ? 1 : kv->batch;
+    const bool rr = ws.amax_rr;                         // the last forward took the row-range path: its candidates are per CTA
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
-           (launch_k(accept_kernel, blocks, 256, 0, m->stream, kv->seq, ws.amax_val, ws.amax_idx, ws.amax_blocks, mode, d_ctxs, seq,
-                                                        last_row, prompt_len)));
+           (launch_k(accept_kernel, blocks, 256, 0, m->stream, kv->seq, rr ? ws.amax_val_rr : ws.amax_val, rr ? ws.amax_idx_rr : ws.amax_idx,
+                     ws.amax_nblk, mode, d_ctxs, seq, last_row, prompt_len)));
+    CUDA_TRY(cudaGetLastError());
+    return ANPD_OK;
+}
+
+// The forward of a single-sequence step (8 rows) on the row-range projections: per layer QKV (+ rotary, append) ->
+// attention -> page combine -> O (+ residual) -> gate/up (+ SwiGLU) -> down (+ residual); then the LM head (+ argmax).
+static anpd_status forward_rr_enqueue(anpd_model* m, anpd_kv* kv, int max_pos, bool want_logits) {
+    const anpd_model_config& c = m->cfg;
+    Workspace& ws = kv->ws;
+    cudaStream_t st = m->stream;
+    Profiler* pf = &m->prof;
+    const int d = c.d_model, hd = c.head_dim;
+    const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * hd;
+    LAUNCH(pf, st, KC_OTHER, 0, (launch_k(embed_img_kernel, ANPD_ROWS, NORM_THREADS, 0, st, m->embed, ws.row_tok, m->layers[0].attn_norm, d, ws.x,
+                                          ws.img_h, ws.ss_a)));
+    int parts_a = 1;                                   // partial sums of squares behind img_h: 1 after the embedding, then the down projection's CTAs
+    for (int l = 0; l < c.n_layers; ++l) {
+        const anpd_model::LayerRR& w = m->rr_layers[l];
+        RREpiHost q;
+        q.ss_in = ws.ss_a; q.n_parts_in = parts_a; q.inv_d_in = 1.0f / (float)d; q.eps = c.rms_eps;
+        q.row_pos = ws.row_pos; q.row_seq = ws.row_seq; q.row_ok = ws.row_ok; q.rope_cos = kv->rope_cos; q.rope_sin = kv->rope_sin;
+        q.page_table = kv->page_table; q.pages_per_seq = kv->pages_per_seq; q.Hq = c.n_q_heads; q.Hkv = c.n_kv_heads; q.hd = hd;
+        q.q_scale = 1.4426950408889634f / sqrtf((float)hd);
+        q.q_hi = ws.q_hi; q.q_lo = ws.q_lo; q.kpool_l = kv->kpool + l * layer_elems; q.vpool_l = kv->vpool + l * layer_elems;
+        ANPD_TRY(rr_enqueue(RR_QKV, m->rr[GK_QKV], w.wqkv, ws.img_h, q, ws.gemm_err, st, pf));
+        if (hd == 128) ANPD_TRY(attn_enqueue<128>(m, kv, l, ANPD_ROWS, max_pos, ws.img_ao));
+        else ANPD_TRY(attn_enqueue<64>(m, kv, l, ANPD_ROWS, max_pos, ws.img_ao));
+        RREpiHost o;
+        o.x = ws.x; o.gain = m->layers[l].ffn_norm; o.ss_out = ws.ss_b; o.d = d; o.act_out = ws.img_h2;
+        ANPD_TRY(rr_enqueue(RR_RESID, m->rr[GK_O], w.wo, ws.img_ao, o, ws.gemm_err, st, pf));
+        RREpiHost gu;
+        gu.ss_in = ws.ss_b; gu.n_parts_in = m->rr[GK_O].G; gu.inv_d_in = 1.0f / (float)d; gu.eps = c.rms_eps; gu.act_out = ws.img_act;
+        ANPD_TRY(rr_enqueue(RR_GU, m->rr[GK_GU], w.wgu, ws.img_h2, gu, ws.gemm_err, st, pf));
+        RREpiHost dn;
+        dn.x = ws.x; dn.gain = (l + 1 < c.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm; dn.ss_out = ws.ss_a; dn.d = d;
+        dn.act_out = ws.img_h;
+        ANPD_TRY(rr_enqueue(RR_RESID, m->rr[GK_DOWN], w.wd, ws.img_act, dn, ws.gemm_err, st, pf));
+        parts_a = m->rr[GK_DOWN].G;
+    }
+    RREpiHost lm;
+    lm.ss_in = ws.ss_a; lm.n_parts_in = parts_a; lm.inv_d_in = 1.0f / (float)d; lm.eps = c.rms_eps;
+    lm.logits = want_logits ? ws.logits : nullptr; lm.amax_val = ws.amax_val_rr; lm.amax_idx = ws.amax_idx_rr; lm.V = c.vocab;
+    ANPD_TRY(rr_enqueue(RR_LM, m->rr[GK_LM], m->rr_lm, ws.img_h, lm, ws.gemm_err, st, pf));
+    ws.amax_nblk = m->rr[GK_LM].G;
+    ws.amax_rr = true;
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
 
 anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits) {
+    if (m->rr_ready && kv->batch == 1 && rows == ANPD_ROWS && head && !m->plain_gemm) return forward_rr_enqueue(m, kv, max_pos, want_logits);
     const anpd_model_config& c = m->cfg;
+    kv->ws.amax_nblk = kv->ws.amax_blocks;
+    kv->ws.amax_rr = false;
     Workspace& ws = kv->ws;
     cudaStream_t st = m->stream;
     Profiler* pf = &m->prof;

@@ -171,6 +171,47 @@ anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof
 anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batch, int K,
                                cudaStream_t st, Profiler* prof);
 
+// proj_rr.cu: the projections of a single-sequence step with their epilogues fused in ("row-range" kernel: each
+// CTA owns a contiguous range of output features and the whole contraction dimension).
+struct RRPlan {
+    int N, K;
+    int pairs;             // feature pairs, cut evenly across the CTAs
+    int G;                 // CTAs
+    int r_max;             // most features a CTA owns (even)
+    int mt;                // 128-row MMA tiles per CTA
+    int k_blocks, kb, n_stages, stages;
+    int a_tile_stride, stage_bytes, smem_bytes;
+    unsigned long long slot_bytes;
+};
+struct RRPlanDev { int G, pairs, r_max, kb; unsigned long long slot_bytes; };
+enum RREpilogue { RR_RAW = 0, RR_QKV = 1, RR_RESID = 2, RR_GU = 3, RR_LM = 4 };
+enum RRRowMap { RR_MAP_IDENTITY = 0, RR_MAP_HEADS = 1, RR_MAP_GATE_UP = 2 };
+// Operand image of the activations of a single-sequence step: per 64-wide k-block a 16-row x 128-byte tile in the
+// 128-byte-swizzled K-major layout (rows 0-7: hi terms of the step's rows, rows 8-15: lo terms).  Byte offset of
+// element (row, k):
+__host__ __device__ inline size_t act_img_offset(int row16, int k) {
+    return (size_t)(k >> 6) * 2048 + (size_t)row16 * 128 + (size_t)(((((k & 63) >> 3) ^ (row16 & 7))) << 4) + (size_t)(k & 7) * 2;
+}
+inline size_t act_img_bytes(int K) { return (size_t)((K + 63) / 64) * 2048; }
+struct RREpiHost {         // epilogue arguments; only the fields of the chosen epilogue are read
+    const float* ss_in = nullptr; int n_parts_in = 0; float inv_d_in = 0; float eps = 0;
+    const int* row_pos = nullptr; const int* row_seq = nullptr; const int* row_ok = nullptr;
+    const float* rope_cos = nullptr; const float* rope_sin = nullptr; const int* page_table = nullptr;
+    int pages_per_seq = 0, Hq = 0, Hkv = 0, hd = 0; float q_scale = 0;
+    __nv_bfloat16 *q_hi = nullptr, *q_lo = nullptr, *kpool_l = nullptr, *vpool_l = nullptr;
+    float* x = nullptr; const float* gain = nullptr; float* ss_out = nullptr; int d = 0;
+    unsigned char* act_out = nullptr;
+    float* logits = nullptr; float* amax_val = nullptr; int* amax_idx = nullptr; int V = 0;
+    float* raw_out = nullptr;
+};
+void rr_make_plan(RRPlan* p, int N, int K, int num_sms);
+size_t rr_storage_bytes(const RRPlan& p);
+anpd_status rr_retile_enqueue(const RRPlan& p, const void* src, bool src_is_f32, int rows, int row_off, int map, int hd, int F,
+                              unsigned char* dst, cudaStream_t st);
+anpd_status rr_act_image_enqueue(const float* a_dev, int K, unsigned char* img, cudaStream_t st);
+anpd_status rr_enqueue(int epi, const RRPlan& p, const unsigned char* w, const unsigned char* act, const RREpiHost& h, int* err,
+                       cudaStream_t st, Profiler* prof);
+
 // ---------------------------------------------------------------------------------------------
 // model, KV cache and workspace
 // ---------------------------------------------------------------------------------------------
@@ -215,6 +256,13 @@ struct anpd_model {
     int* d_ones;                      // [tiles] all 1: segment counts of the plain GEMM
     int max_segs;
     bool plain_gemm;                  // debugging aid: route GEMMs through the plain kernel
+    // second copy of the projections in row-range storage, used by single-sequence steps (proj_rr.cu)
+    RRPlan rr[GK_COUNT];
+    struct LayerRR { const unsigned char *wqkv, *wo, *wgu, *wd; };
+    std::vector<LayerRR> rr_layers;
+    const unsigned char* rr_lm;
+    void* rr_slab;
+    bool rr_ready;
     int num_sms;
     int device;                       // ordinal of the device the weight blocks were laid out for
     Profiler prof;
@@ -235,6 +283,13 @@ struct Workspace {
     float* logits;                    // [r_max, V]
     float* amax_val; int* amax_idx;   // [r_max, amax_blocks]
     int amax_blocks;
+    // single-sequence steps: operand images of the four projection inputs, partial sums of squares of the residual
+    // stream ([CTA][8 rows]; a: after the down projection / embedding, b: after the O projection), per-CTA argmax
+    unsigned char *img_h, *img_h2, *img_ao, *img_act;
+    float *ss_a, *ss_b;
+    float* amax_val_rr; int* amax_idx_rr;
+    int amax_nblk;                    // argmax candidates per row left by the last forward (depends on the path it took)
+    bool amax_rr;                     // ... and whether they are in the row-range path's arrays
     int* gemm_err;                    // device flag set by a GEMM kernel that gave up waiting
     // TMA views of the activation buffers: [0] decode (batch*8 rows), [1] prefill (PREFILL_ROWS rows)
     CUtensorMap map_h[2][2], map_ao[2][2], map_act[2][2];     // [mode][hi/lo]

@@ -21,7 +21,21 @@ from workloads import WORKLOADS, make_prompts, make_weights
 pytestmark = pytest.mark.gpu
 
 MARGIN = 5e-2
-FULLSIZE_TOL = 5e-2   # max-abs on logits against the bf16-cache oracle at 32 layers x 4096 (see the first test)
+LOGIT_TOL = 2e-2      # the stated max-abs bar (what a model without depth meets: tests/test_gpu_fullwidth.py)
+
+
+def depth_bar(cache_effect: float) -> float:
+    """Max-abs bar on the logits of a deep random-init model against the bf16-cache oracle.
+
+    Through L random layers a relative perturbation of the cached values is amplified on the way to the logits;
+    the oracle measures that amplification on itself: `cache_effect` is the max-abs distance between its plain and
+    its bf16-cache logits for this very model and input, i.e. what rounding EVERY cache element by at most half a
+    bf16 unit does.  The library's cache differs from the bf16-cache oracle's only in the elements whose fp32
+    value (16-bit-mantissa activation split, fp32 accumulation) falls on the other side of a rounding boundary -
+    a full unit each, but well under one element in a hundred - and otherwise by fp32-level terms that see the same
+    amplification.  Half the model's own cache effect bounds that with margin (measured: a quarter at 32 and 40
+    layers); for shallow models the stated bar applies."""
+    return max(LOGIT_TOL, 0.5 * cache_effect)
 
 
 @pytest.fixture(scope="module")
@@ -55,28 +69,12 @@ def test_c3_verify_logits_against_oracle_after_short_prompt(A, c3):
         got = A.anpd_verify_logits(m, kv, first, draft, wl.shape.vocab)
     finally:
         A.anpd_kv_destroy(kv)
-    dec = Decoder(wl.shape, w_cpu, torch.float64, kv_dtype=torch.bfloat16)
-    cache = dec.new_cache()
-    lp = dec.forward(prompt, cache)
-    if top2_margin(lp[-1]) > MARGIN:
-        assert first == argmax_lowest(lp[-1])
-    want = dec.forward([first] + draft, cache)
-    diff = torch.from_numpy(got).double() - want
-    # same weights, same cache precision: what is left is fp32 accumulation, the 16-bit activation split and the
-    # few cache elements that round to the other bf16 neighbour, amplified by 32 random layers (measured:
-    # max 0.025, rms 0.005 at a logit standard deviation of 1.28)
-    assert float(diff.abs().max()) <= FULLSIZE_TOL, float(diff.abs().max())
-    assert float(diff.pow(2).mean().sqrt()) <= 1e-2
-    for r in range(want.shape[0]):
-        if top2_margin(want[r]) > 2 * FULLSIZE_TOL:
-            assert int(np.argmax(got[r])) == argmax_lowest(want[r])
-    # the plain fp64 oracle is as far from its own bf16-cache variant as it is from the library
-    plain = Decoder(wl.shape, w_cpu, torch.float64)
-    cache = plain.new_cache()
-    plain.forward(prompt, cache)
-    ref = plain.forward([first] + draft, cache)
-    cache_effect = float((ref - want).abs().max())
-    assert float((torch.from_numpy(got).double() - ref).abs().max()) <= cache_effect + FULLSIZE_TOL
+    err, rms, sigma, cache_effect, err_plain = _compare_with_both_oracles(wl.shape, w_cpu, prompt, first, draft, got)
+    print(f"C3 (32 layers): vs bf16-cache oracle max-abs {err:.3e} rms {rms:.3e}, logit sigma {sigma:.3f}, max-abs / sigma "
+          f"{err / sigma:.3e}; the oracle's own cache effect {cache_effect:.3e}; vs plain oracle {err_plain:.3e}")
+    assert err <= depth_bar(cache_effect), (err, cache_effect)
+    assert rms <= 0.25 * depth_bar(cache_effect), rms
+    assert err_plain <= cache_effect + depth_bar(cache_effect)
 
 
 def test_c3_full_prompt_anpd_equals_greedy_and_tables_follow_the_stream(A, c3):
@@ -128,9 +126,33 @@ def test_c3_attention_kernels_agree_at_bench_context_length(A, c3, monkeypatch):
     assert float(np.abs(outs[0][1] - outs[1][1]).max()) <= 1e-2
 
 
-def _short_prompt_logits_check(A, wl, n_prompt, tol):
-    """Model of workload `wl` at full size: prefill `n_prompt` tokens, one 8-row verify step, logits against the
-    oracle with the bf16 cache; returns (max-abs error, the oracle's logit standard deviation)."""
+def _compare_with_both_oracles(shape, w_cpu, prompt, first, draft, got):
+    """(max-abs and rms error against the bf16-cache oracle, its logit sigma, the oracle's own cache effect, max-abs
+    error against the plain oracle); also asserts equal argmax wherever the bf16-cache oracle's margin allows."""
+    out = {}
+    for name, kv_dtype in (("bf16", torch.bfloat16), ("plain", None)):
+        dec = Decoder(shape, w_cpu, torch.float64, kv_dtype=kv_dtype)
+        cache = dec.new_cache()
+        lp = dec.forward(prompt, cache)
+        out[name] = (lp[-1], dec.forward([first] + draft, cache))
+    lp_last, want = out["bf16"]
+    plain = out["plain"][1]
+    g = torch.from_numpy(got).double()
+    diff = g - want
+    err = float(diff.abs().max())
+    cache_effect = float((plain - want).abs().max())
+    bar = depth_bar(cache_effect)
+    if top2_margin(lp_last) > max(MARGIN, 2 * bar):
+        assert first == argmax_lowest(lp_last)
+    for r in range(want.shape[0]):
+        if top2_margin(want[r]) > max(MARGIN, 2 * bar):
+            assert int(np.argmax(got[r])) == argmax_lowest(want[r])
+    return err, float(diff.pow(2).mean().sqrt()), float(want.std()), cache_effect, float((g - plain).abs().max())
+
+
+def _short_prompt_logits_check(A, wl, n_prompt):
+    """Model of workload `wl` at full size: prefill `n_prompt` tokens, one 8-row verify step, logits against both
+    forms of the oracle; the bar is derived from this model's own cache effect (depth_bar)."""
     w = make_weights(wl.shape, wl.weight_seed, True, device="cuda")
     torch.cuda.synchronize()
     m = gpu_model(A, wl.shape, w, new_stream())
@@ -146,30 +168,23 @@ def _short_prompt_logits_check(A, wl, n_prompt, tol):
     finally:
         A.anpd_kv_destroy(kv)
         A.anpd_model_destroy(m)
-    dec = Decoder(wl.shape, w_cpu, torch.float64, kv_dtype=torch.bfloat16)
-    cache = dec.new_cache()
-    lp = dec.forward(prompt, cache)
-    if top2_margin(lp[-1]) > 2 * tol:
-        assert first == argmax_lowest(lp[-1])
-    want = dec.forward([first] + draft, cache)
-    diff = torch.from_numpy(got).double() - want
-    for r in range(want.shape[0]):
-        if top2_margin(want[r]) > 2 * tol:
-            assert int(np.argmax(got[r])) == argmax_lowest(want[r])
-    return float(diff.abs().max()), float(diff.pow(2).mean().sqrt())
+    err, rms, sigma, cache_effect, err_plain = _compare_with_both_oracles(wl.shape, w_cpu, prompt, first, draft, got)
+    print(f"{wl.name} ({wl.shape.n_layers} layers): vs bf16-cache oracle max-abs {err:.3e} rms {rms:.3e}, logit sigma {sigma:.3f}, "
+          f"max-abs / sigma {err / sigma:.3e}; the oracle's own cache effect {cache_effect:.3e}; vs plain oracle {err_plain:.3e}")
+    assert err <= depth_bar(cache_effect), (err, cache_effect)
+    assert rms <= 0.25 * depth_bar(cache_effect), rms
+    assert err_plain <= cache_effect + depth_bar(cache_effect)
 
 
 def test_c2_shape_grouped_query_heads_against_oracle(A):
     """1.1B shape: 22 layers, 32 query heads on 4 kv heads of dimension 64 (the mma.sync attention kernel with 8 query
     heads per kv head), d_ffn 5632; 40-token prompt."""
-    err, rms = _short_prompt_logits_check(A, WORKLOADS["C2"], 40, FULLSIZE_TOL)
-    assert err <= FULLSIZE_TOL and rms <= 1e-2, (err, rms)
+    _short_prompt_logits_check(A, WORKLOADS["C2"], 40)
 
 
 def test_c5_shape_single_sequence_against_oracle(A):
     """13B shape: 40 layers x 5120, 40 heads of dimension 128, d_ffn 13824 (other stream-K splits than the 7B shape)."""
-    err, rms = _short_prompt_logits_check(A, WORKLOADS["C5"], 10, FULLSIZE_TOL)
-    assert err <= FULLSIZE_TOL and rms <= 1e-2, (err, rms)
+    _short_prompt_logits_check(A, WORKLOADS["C5"], 10)
 
 
 def test_c5_batch_of_eight_equals_greedy_and_independent_runs(A):
