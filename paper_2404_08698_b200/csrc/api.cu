@@ -61,6 +61,13 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restri
         dst[i] = __float2bfloat16_rn(src[i]);
 }
 __global__ void set_int_kernel(int* p, int v) { *p = v; }
+// A sequence that starts over: empty cache, counters cleared, active (a finished decoding loop leaves it retired).
+__global__ void seq_restart_kernel(SeqState* s) {
+    s->kv_len = 0; s->draft_len = 0; s->accepted_len = 0;
+    s->steps = 0; s->drafted = 0; s->accepted = 0;
+    for (int i = 0; i < 8; ++i) s->hist[i] = 0;
+    s->active = 1; s->stop_at = 0x7fffffff; s->error = 0;
+}
 __global__ void greedy_stage_kernel(SeqState* seqs) {
     pdl_trigger();
     pdl_wait();
@@ -527,6 +534,8 @@ anpd_status anpd_prefill(anpd_model* m, anpd_kv* kv, int seq, const int32_t* pro
     if (kv->h_kv_len[seq] != 0) return ANPD_ERR_STATE;
     if (prompt_len + ANPD_ROWS > kv->max_len) return ANPD_ERR_CAPACITY;
     for (int i = 0; i < prompt_len; ++i) if (prompt[i] < 0 || prompt[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+    LAUNCH(&m->prof, m->stream, KC_OTHER, 0, (seq_restart_kernel<<<1, 1, 0, m->stream>>>(&kv->seq[seq])));
+    CUDA_TRY(cudaGetLastError());
     ANPD_TRY(prefill_enqueue(m, kv, seq, prompt, prompt_len, nullptr));
     ANPD_TRY(read_seqs(kv));
     ANPD_TRY(seq_error_status(kv->h_seq[seq]));

@@ -178,21 +178,27 @@ struct RRPlan {
     int pairs;             // feature pairs, cut evenly across the CTAs
     int G;                 // CTAs
     int r_max;             // most features a CTA owns (even)
-    int mt;                // 128-row MMA tiles per CTA
+    int mt;                // features per epilogue thread (1 or 2)
+    int P;                 // 16-wide slices of K packed into one MMA (1, 2, 4 or 8; P * r_max <= 256)
     int k_blocks, kb, n_stages, stages;
-    int a_tile_stride, stage_bytes, smem_bytes;
+    int w_step_stride, w_step_global, a_off, stage_bytes, scratch_off, smem_bytes;
+    int rotate, one_copy;
     unsigned long long slot_bytes;
 };
-struct RRPlanDev { int G, pairs, r_max, kb; unsigned long long slot_bytes; };
+struct RRPlanDev { int G, pairs, r_max, kb, n_stages, rotate, P, w_step_global; unsigned long long slot_bytes; };
+// Stage at which CTA c of G starts its walk over the n_stages stages of K (it wraps around).
+__host__ __device__ inline int rr_rotation(int c, int G, int n_stages) { return (int)((long long)c * n_stages / G); }
 enum RREpilogue { RR_RAW = 0, RR_QKV = 1, RR_RESID = 2, RR_GU = 3, RR_LM = 4 };
 enum RRRowMap { RR_MAP_IDENTITY = 0, RR_MAP_HEADS = 1, RR_MAP_GATE_UP = 2 };
-// Operand image of the activations of a single-sequence step: per 64-wide k-block a 16-row x 128-byte tile in the
-// 128-byte-swizzled K-major layout (rows 0-7: hi terms of the step's rows, rows 8-15: lo terms).  Byte offset of
-// element (row, k):
+// Operand image of the activations of a single-sequence step: per 64-wide k-block 64 operand rows of 32 bytes
+// (row = 16 * slice + term, slice = the 16-wide part of the k-block, terms 0-7 = hi parts of the step's rows, 8-15 = lo
+// parts) in the 32-byte-swizzled K-major layout.  Byte offset of element (term row16, k):
 __host__ __device__ inline size_t act_img_offset(int row16, int k) {
-    return (size_t)(k >> 6) * 2048 + (size_t)row16 * 128 + (size_t)(((((k & 63) >> 3) ^ (row16 & 7))) << 4) + (size_t)(k & 7) * 2;
+    const int R = ((k >> 4) & 3) * 16 + row16;
+    return (size_t)(k >> 6) * 2048 + (size_t)R * 32 + (size_t)(((((k >> 3) & 1) ^ ((R >> 2) & 1))) << 4) + (size_t)(k & 7) * 2;
 }
-inline size_t act_img_bytes(int K) { return (size_t)((K + 63) / 64) * 2048; }
+// one k-block more than K needs, left zero: an instruction that packs eight slices spans two k-blocks
+inline size_t act_img_bytes(int K) { return (size_t)((K + 63) / 64 + 1) * 2048; }
 struct RREpiHost {         // epilogue arguments; only the fields of the chosen epilogue are read
     const float* ss_in = nullptr; int n_parts_in = 0; float inv_d_in = 0; float eps = 0;
     const int* row_pos = nullptr; const int* row_seq = nullptr; const int* row_ok = nullptr;
