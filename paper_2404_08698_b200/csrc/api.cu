@@ -219,8 +219,9 @@ anpd_status anpd_model_create(const anpd_model_config* cfg, const void* const* w
     }
     m->rr_slab = nullptr;
     m->rr_lm = nullptr;
-    // single-sequence steps run on a second copy of the projections in row-range storage (ANPD_NO_RR=1: stream-K only)
-    m->rr_ready = std::getenv("ANPD_NO_RR") == nullptr;
+    // ANPD_RR=1: single-sequence steps run on a second copy of the projections in row-range storage (proj_rr.cu).  Off
+    // by default: measured at every model shape, the fused epilogues cost more than the small kernels they replace.
+    m->rr_ready = std::getenv("ANPD_RR") != nullptr;
     for (int k = 0; k < GK_COUNT; ++k)
         if (m->rr[k].mt > 2) m->rr_ready = false;      // a CTA's feature range must fit two 128-row MMA tiles (very large vocabularies do not)
     const size_t b_embed = up256(V * d * 2), b_lm = up256(gemm_tiled_elems(m->plan[GK_LM]) * 2),

@@ -282,3 +282,30 @@ def test_long_context_attention_slots_take_several_pages(A, monkeypatch):
     want = dec.forward([outs[0][0]] + draft, cache)
     err = float((torch.from_numpy(outs[0][1]).double() - want).abs().max())
     assert err <= LOGIT_TOL, err
+
+
+@pytest.mark.parametrize("shape,plen", [(ModelShape(2, 256, 4, 4, 64, 688, 4096), 140),      # the tiny workload's shape
+                                        (ModelShape(2, 512, 4, 2, 128, 1000, 3001), 300),    # hd 128, grouped heads, odd vocabulary, ragged K
+                                        (ModelShape(1, 1024, 8, 1, 128, 2816, 5000), 90)])   # 8 query heads per kv head
+def test_row_range_projections_logits_parity(A, monkeypatch, shape, plen):
+    """The optional single-sequence path (ANPD_RR=1: projections with rotary/append, residual + deferred RMSNorm, SwiGLU
+    and the vocabulary argmax fused into their epilogues) against the oracle, same bars as the default path."""
+    monkeypatch.setenv("ANPD_RR", "1")
+    r = Rig(A, shape, seed=31, jitter=0.1)
+    try:
+        prompt = markov_prompt(plen, shape.vocab, 2, 77).tolist()
+        first = A.anpd_prefill(r.m, r.kv, prompt)
+        draft = [int(t) for t in prompt[5:12]]
+        got = A.anpd_verify_logits(r.m, r.kv, first, draft, shape.vocab)
+        cache = r.dec.new_cache()
+        r.dec.forward(prompt, cache)
+        want = r.dec.forward([first] + draft, cache)
+        err = float((torch.from_numpy(got).double() - want).abs().max())
+        assert err <= LOGIT_TOL, err
+        # and the committing step takes the decisions the logits imply
+        acc, nxt = A.anpd_verify(r.m, r.kv, first, draft)
+        preds = [int(np.argmax(got[i])) for i in range(8)]
+        assert acc == accept_length(draft, preds) and nxt == preds[acc]
+        assert A.anpd_kv_len(r.kv) == plen + acc + 1
+    finally:
+        r.close()

@@ -64,3 +64,43 @@ def test_periodic_prompt():
     p = periodic_prompt(40, 7, 100, 3)
     assert len(set(p[:7].tolist())) == 7
     assert all(p[i] == p[i % 7] for i in range(40))
+
+
+# ---- orbit workloads: a model with a closed-form continuation -------------------------------------
+def test_orbit_permutation_is_one_cycle_and_prompt_replays_it():
+    from workloads import orbit_continuation, orbit_permutation, orbit_prompt
+    pi = orbit_permutation(97, 5)
+    assert sorted(pi.tolist()) == list(range(97))
+    t, n = 0, 0
+    while True:
+        t, n = int(pi[t]), n + 1
+        if t == 0:
+            break
+    assert n == 97                                              # a single cycle through every token
+    p = orbit_prompt(pi, 60, 0.0, 3)
+    assert all(int(pi[p[i]]) == p[i + 1] for i in range(58))    # uncorrupted: the orbit itself
+    assert p[-1] == p[8]                                        # closed by its own ninth token
+    assert orbit_continuation(pi, p[-1], 20).tolist() == p[9:29].tolist()
+    q = orbit_prompt(pi, 60, 0.5, 3)
+    assert 10 < int((q[:-1] != p[:-1]).sum()) < 45 and q[:9].tolist() == p[:9].tolist()
+
+
+def test_orbit_model_continues_its_orbit_under_the_oracle_decoder():
+    """The real decoder on the orbit weights decodes exactly the closed-form continuation, and the scripted stand-in
+    takes the same ANPD steps (it is what the full-size GPU tests compare their statistics with)."""
+    import torch
+    from oracle.anpd import anpd_generate, greedy
+    from oracle.decoder import Decoder
+    from workloads import WORKLOADS, ScriptedOrbitModel, orbit_permutation, workload_inputs
+    wl = WORKLOADS["C1-A50"]
+    w, prompts, expected = workload_inputs(wl)
+    dec = Decoder(wl.shape, w, torch.float64)
+    prompt = prompts[0].tolist()
+    assert greedy(dec, prompt, 24) == expected[0][:24].tolist()
+    out, st, _ = anpd_generate(dec, prompt, wl.max_new, wl.K, n_max=wl.n_max)
+    pi = orbit_permutation(wl.orbit_S, wl.weight_seed)
+    out2, st2, _ = anpd_generate(ScriptedOrbitModel(pi, wl.shape.vocab), prompt, wl.max_new, wl.K, n_max=wl.n_max)
+    assert out == out2 == expected[0][:wl.max_new].tolist()
+    assert (st.steps, st.drafted, st.accepted, st.hist_accepted, st.drafts, st.accepted_lens) == \
+           (st2.steps, st2.drafted, st2.accepted, st2.hist_accepted, st2.drafts, st2.accepted_lens)
+    assert 0.3 < st.hit_ratio < 0.8

@@ -56,6 +56,10 @@ class Workload:
     batch: int = 1
     prompt_seed: int = 1000
     n_min: int = 2
+    # orbit workloads (workloads/orbit.py): a model whose greedy continuation is known, and a prompt that makes the
+    # n-gram drafts right part of the time; orbit_S = 0 means the ordinary random-init model and Markov prompt
+    orbit_S: int = 0
+    corrupt: float = 0.0
 
 
 TINY = ModelShape(2, 256, 4, 4, 64, 688, 4096)
@@ -69,6 +73,13 @@ WORKLOADS = {
     "C3": Workload("C3", S7B, True, 2, 1536, 3, True, 256, 5, 5, 1, 1002),
     # C4 (verify-step microbenchmark) reuses the C3 model; see bench.py
     "C5": Workload("C5", S13B, True, 3, 2048, 3, True, 512, 7, 6, 8, 1004),
+    # The 7B shape with a controlled answer (orbit model, same byte traffic as C3): prompts whose n-gram drafts hit about
+    # 20 % / 60 % of the time (the paper's case study reports a hit ratio of 20.59 %, Section 4.4).
+    "C3-A20": Workload("C3-A20", S7B, True, 2, 1536, 3, False, 256, 5, 5, 1, 1012, orbit_S=4096, corrupt=0.39),
+    "C3-A60": Workload("C3-A60", S7B, True, 2, 1536, 3, False, 256, 5, 5, 1, 1013, orbit_S=4096, corrupt=0.15),
+    # the same construction at the 1.1B shape and at a size the oracle's full decoder runs in seconds
+    "C2-A40": Workload("C2-A40", S1B, True, 1, 512, 3, False, 256, 5, 5, 1, 1014, orbit_S=2048, corrupt=0.25),
+    "C1-A50": Workload("C1-A50", TINY, False, 0, 128, 2, False, 64, 3, 4, 1, 1015, orbit_S=256, corrupt=0.2),
     # two layers of the 7B shape: the per-layer kernels of C3 at a size a profiler capture can hold
     "C3-2L": Workload("C3-2L", ModelShape(2, 4096, 32, 32, 128, 11008, 32000), True, 2, 1536, 3, True, 256, 5, 5, 1, 1002),
 }
