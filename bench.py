@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from workloads import WORKLOADS, make_prompts, make_weights, tensor_shapes
+from workloads import WORKLOADS, make_prompts, make_weights, tensor_shapes, workload_inputs
 
 METRIC = "tokens_per_s_bs1_anpd"
 UNIT = "tokens/s"
@@ -100,17 +100,61 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(wl, weights_cpu, prompt, sample_prompt: int, sample_new: int) -> dict:
-    """Times the CPU oracle (as it stands) on a bounded sample of the workload."""
-    from oracle.anpd import anpd_generate as oracle_anpd
+def oracle_baseline(wl, weights_cpu, prompt, mean_accepted: float | None = None, budget_s: float = 60.0) -> dict:
+    """The CPU oracle, as it stands, timed on this machine's host cores on a bounded sample of the workload.
+
+    The oracle runs in its fp32 mode with every weight cast once (same arithmetic, see oracle/decoder.py).  Small
+    workloads (below 3 G streamed parameters) are run whole: the oracle's greedy decode and its Algorithm 1, which
+    gives the oracle's own ANPD / greedy ratio.  For the large ones the prompt is prefilled once (so that the timed
+    forwards see the workload's own KV length) and then >= 3 verify forwards of width K+1 and >= 3 single-token
+    greedy forwards are timed; tokens/s follow from those."""
+    from oracle.anpd import anpd_generate as oracle_anpd, greedy as oracle_greedy, verify as oracle_verify
     from oracle.decoder import Decoder
-    dec = Decoder(wl.shape, weights_cpu, torch.float64)
+    cores = os.cpu_count() or 0
+    threads = torch.get_num_threads()
+    dec = Decoder(wl.shape, weights_cpu, torch.float32, keep_cast=True)
+    base = {"unit": UNIT, "cores": threads, "host_cpus": cores, "kind": "oracle", "dtype": "f32"}
+    toks = prompt.tolist()
+    if wl.shape.streamed_params < 3e9:
+        t0 = time.perf_counter()
+        g = oracle_greedy(dec, toks, wl.max_new)
+        t_g = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        out, st, _ = oracle_anpd(dec, toks, wl.max_new, wl.K, n_max=wl.n_max, n_min=wl.n_min)
+        t_a = time.perf_counter() - t0
+        base.update({"value": wl.max_new / t_a, "greedy_tokens_per_s": wl.max_new / t_g, "anpd_over_greedy": t_g / t_a,
+                     "hit_ratio_alpha": st.hit_ratio, "steps": st.steps, "anpd_equals_greedy": out == g,
+                     "sample": f"the whole workload {wl.name} on the oracle (fp32 torch CPU ops, weights cast once): greedy decode "
+                               f"{t_g:.1f} s, Algorithm 1 {t_a:.1f} s (prompt {len(toks)}, {wl.max_new} new tokens, N={wl.n_max}, K={wl.K})"})
+        return base
+    if wl.shape.streamed_params > 1e10:                 # 13B shape: bound the prefill of the sample
+        toks = toks[:256]
+    cache = dec.new_cache()
     t0 = time.perf_counter()
-    out, st, _ = oracle_anpd(dec, prompt[:sample_prompt].tolist(), sample_new, wl.K, n_max=wl.n_max, n_min=wl.n_min)
-    dt = time.perf_counter() - t0
-    return {"value": len(out) / dt, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-            "sample": f"oracle Algorithm 1 (fp64 torch CPU ops) on the first {sample_prompt} prompt tokens of {wl.name}, "
-                      f"{sample_new} new tokens, N={wl.n_max}, K={wl.K}: {st.steps} verify forwards + 1 prefill in {dt:.1f} s"}
+    logits = dec.forward(toks, cache)
+    t_prefill = time.perf_counter() - t0
+    first = int(torch.argmax(logits[-1]))
+    P = cache.length
+    draft = [int(t) for t in toks[:wl.K]]
+    tv, tg = [], []
+    for _ in range(3):
+        t0 = time.perf_counter()
+        oracle_verify(dec, cache, first, draft)
+        tv.append(time.perf_counter() - t0)
+        cache.truncate(P)
+    for _ in range(3):
+        t0 = time.perf_counter()
+        dec.forward([first], cache)
+        tg.append(time.perf_counter() - t0)
+        cache.truncate(P)
+    t_v, t_g = statistics.median(tv), statistics.median(tg)
+    acc = 0.0 if mean_accepted is None else mean_accepted
+    base.update({"value": (1.0 + acc) / t_v, "greedy_tokens_per_s": 1.0 / t_g, "verify_forward_s": t_v, "greedy_forward_s": t_g,
+                 "prefill_s": t_prefill, "kv_len": P,
+                 "sample": f"oracle (fp32 torch CPU ops, weights cast once) on {wl.name}: one prefill of the {len(toks)}-token prompt "
+                           f"({t_prefill:.1f} s, untimed in the value), then 3 verify forwards of width K+1={wl.K + 1} and 3 single-token "
+                           f"greedy forwards at KV {P}; value = (1 + mean accepted per step {acc:.2f}) / median verify forward"})
+    return base
 
 
 def run_reference(args) -> None:
@@ -120,26 +164,21 @@ def run_reference(args) -> None:
         return
     wl = WORKLOADS[args.workload]
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    w = make_weights(wl.shape, wl.weight_seed, wl.weights_bf16, device=dev)
+    w, prompts, _ = workload_inputs(wl, device=dev)
     w = {k: v.cpu() for k, v in w.items()}
-    prompt = make_prompts(wl)[0]
-    big = wl.shape.streamed_params > 3e9
-    sp, sn = (16, 2) if big else ((64, 8) if wl.shape.streamed_params > 1e8 else (wl.prompt_len, wl.max_new))
-    for _ in range(args.warmup):
-        oracle_sample(wl, w, prompt, sp, 1)
+    prompt = prompts[0]
+    res = None
     t0 = time.perf_counter()
-    res = [oracle_sample(wl, w, prompt, sp, sn) for _ in range(args.steps)]
+    for _ in range(max(args.steps, 1) if wl.shape.streamed_params < 1e8 else 1):     # the large workloads: one bounded sample
+        res = oracle_baseline(wl, w, prompt)
     dt = time.perf_counter() - t0
-    value = args.steps * sn / dt
-    cpu = dict(res[-1])
-    cpu["value"] = value
+    value = res["value"]
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{wl.name} (bounded sample: first {sp} prompt tokens, {sn} new tokens per step)",
-                   "n_max": wl.n_max, "K": wl.K},
-        "cpu_baseline": cpu,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{wl.name} (bounded sample, see cpu_baseline.sample)", "n_max": wl.n_max, "K": wl.K},
+        "cpu_baseline": res,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
@@ -168,7 +207,7 @@ def verify_microbench(args, A, wl, model, stream) -> None:
                     for i in range(k):                      # untimed dry runs, one per draft position
                         logits = A.anpd_verify_logits(model, kv, first, draft, shape.vocab)
                         pred = int(np.argmax(logits[i]))
-                        keep = uniform_at(977 + ds, width * 16 + int(p * 100), i) < p
+                        keep = uniform_at(977 + ds + 131 * kv_len, width * 16 + int(p * 100), i) < p
                         draft.append(pred if keep else (pred + 1) % shape.vocab)
                     A.anpd_verify_stage(model, kv, [first], [draft])
                     for _ in range(3):
@@ -201,7 +240,7 @@ def verify_microbench(args, A, wl, model, stream) -> None:
                       "rows": rows_out}))
 
 
-def batch_generate_bench(args, A, wl, model, stream, t_setup0: float) -> None:
+def batch_generate_bench(args, A, wl, model, stream, t_setup0: float, prompts_all, w_cpu) -> None:
     """Workloads with several independent sequences (C5): every verify step carries 8 rows per sequence,
     each sequence has its own n-gram tables, KV pages, draft and acceptance; one weight stream serves
     all of them.  Timed through the host-buffer call (the only batched entry point), with CUDA events
@@ -210,7 +249,7 @@ def batch_generate_bench(args, A, wl, model, stream, t_setup0: float) -> None:
     max_len = wl.prompt_len + wl.max_new + 64
     kv = A.anpd_kv_create(model, max_len, B)
     ctxs = [A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, stream.cuda_stream) for _ in range(B)]
-    prompts = np.stack(make_prompts(wl))
+    prompts = np.stack(prompts_all)
     torch.cuda.synchronize()
     t_setup = time.perf_counter() - t_setup0
 
@@ -259,15 +298,132 @@ def batch_generate_bench(args, A, wl, model, stream, t_setup0: float) -> None:
         "anpd_equals_greedy": bool(np.array_equal(out_anpd, out_greedy)),
         "setup_s": t_setup,
     }
+    # ---- verify step alone and the dominant kernel, at the end-of-run KV lengths ------------------------------------
+    lens = [A.anpd_kv_len(kv, b) for b in range(B)]
+    last = [int(x) for x in out_anpd[:, -1]]
+    drafts = [[int(t) for t in prompts[b][:wl.K]] for b in range(B)]
+    A.anpd_verify_stage(model, kv, last, drafts)
+
+    def one_step():
+        A.anpd_verify_enqueue(model, kv)
+        for b in range(B):
+            A.anpd_kv_truncate(kv, b, lens[b])
+
+    for _ in range(3):
+        one_step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.verify_iters):
+        one_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_verify = e0.elapsed_time(e1) / args.verify_iters
+    step_bytes = shape.streamed_params * 2 + shape.kv_bytes_per_token * sum(l + A.ROWS for l in lens)
+    peak, peak_kind = measured_hbm_peak()
+    A.anpd_profile_enable(model, True)
+    A.anpd_profile_read(model, True)
+    for _ in range(3):
+        one_step()
+    prof = A.anpd_profile_read(model, True)
+    A.anpd_profile_enable(model, False)
+    gemm_gbs = prof["gemm_bytes"] / (prof["ms_gemm"] * 1e-3) / 1e9 if prof["ms_gemm"] > 0 else 0.0
+    result["verify_step"] = {"kv_len": lens, "rows": A.ROWS * B, "ms": ms_verify, "bytes": step_bytes, "gbs": step_bytes / (ms_verify * 1e-3) / 1e9,
+                             "frac_of_8TBs": step_bytes / (ms_verify * 1e-3) / 1e9 / HBM_NOMINAL_GBS,
+                             f"frac_of_{peak_kind}_copy": step_bytes / (ms_verify * 1e-3) / 1e9 / peak}
+    result["roofline"] = {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections + LM head)", "achieved": gemm_gbs, "peak": peak,
+                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": gemm_gbs / peak, "traffic": gemm_traffic_per_launch(wl),
+                          "launches": prof["n_gemm"], "avg_launch_us": prof["ms_gemm"] * 1e3 / max(prof["n_gemm"], 1),
+                          "bytes_per_launch": prof["gemm_bytes"] / max(prof["n_gemm"], 1)}
+    if w_cpu is not None:
+        result["cpu_baseline"] = oracle_baseline(wl, w_cpu, prompts[0], acc / max(steps_sum, 1))
     print(json.dumps(result))
     for c in ctxs:
         A.anpd_ngram_destroy(c)
     A.anpd_kv_destroy(kv)
 
 
-# Mean DRAM bytes (read + write) per weight-GEMM launch of one verify step, from the ncu capture summarised in
-# profiles/gemm_tc_kernel_7B_2layer_ncu.md (one layer's four projections and the LM head, scaled to 32 layers).
-NCU_GEMM_TRAFFIC_PER_LAUNCH = {"C3": 105.5e6}
+def gemm_traffic_per_launch(wl) -> float | None:
+    """Mean DRAM bytes (read + write) per weight-GEMM launch of one verify step of the 7B shape, computed from the
+    committed ncu summary of the GEMM kernel on the two-layer model of that shape (one layer's four projections and the
+    LM head; a full step is n_layers such layers + the LM head, and traffic is proportional to the weights).  None for
+    other shapes, and None if the summary cannot be read."""
+    if wl.shape.d_model != 4096 or wl.shape.d_ffn != 11008 or wl.shape.vocab != 32000:
+        return None
+    try:
+        text = open(os.path.join(ROOT, "profiles", "gemm_tc_kernel_7B_2layer_ncu.md")).read()
+        def row(name):
+            line = next(l for l in text.splitlines() if l.startswith(name))
+            return [float(x) for x in line.split(":", 1)[1].split(",")]
+        rd, wr = row("dram__bytes_read.sum [Mbyte]"), row("dram__bytes_write.sum [Mbyte]")
+        per = [(a + b) * 1e6 for a, b in zip(rd, wr)]          # QKV, O, gate/up, down, LM head
+        L = wl.shape.n_layers
+        return (L * sum(per[:4]) + per[4]) / (4 * L + 1)
+    except Exception:
+        return None
+
+
+def structured_acceptance(args, A, stream, names) -> list:
+    """ANPD against the same build's greedy decode on orbit workloads (workloads/orbit.py): the shape and the bytes
+    streamed per step are the random model's, but the model's continuation is one the n-gram drafts hit part of the time,
+    so the speed-up the method exists for shows.  One model serves all `names` (they differ in their prompts)."""
+    rows = []
+    wl0 = WORKLOADS[names[0]]
+    w, _, _ = workload_inputs(wl0, device="cuda")
+    torch.cuda.synchronize()
+    model = A.anpd_model_create(wl0.shape, [w[n] for n, _ in tensor_shapes(wl0.shape)], stream.cuda_stream)
+    del w
+    torch.cuda.empty_cache()
+    max_len = wl0.prompt_len + wl0.max_new + 64
+    kv = A.anpd_kv_create(model, max_len)
+    ctx = A.anpd_ngram_create(wl0.n_min, wl0.n_max, max_len, 0, stream.cuda_stream)
+    out_dev = torch.zeros(wl0.max_new, dtype=torch.int32, device="cuda")
+    for name in names:
+        wl = WORKLOADS[name]
+        assert wl.shape == wl0.shape and wl.weight_seed == wl0.weight_seed and wl.orbit_S == wl0.orbit_S
+        from workloads import orbit_continuation, orbit_permutation, orbit_prompt
+        pi = orbit_permutation(wl.orbit_S, wl.weight_seed)
+        prompt = orbit_prompt(pi, wl.prompt_len, wl.corrupt, wl.prompt_seed)
+        want = orbit_continuation(pi, prompt[-1], wl.max_new)
+        prompt_dev = torch.from_numpy(prompt).cuda()
+
+        def timed(K):
+            st = None
+            for _ in range(2):
+                st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / 1e3 / args.steps, st, out_dev.cpu().numpy().copy()
+
+        t_a, st_a, out_a = timed(wl.K)
+        t_g, st_g, out_g = timed(0)
+        t0 = time.perf_counter()
+        out_h, _ = A.anpd_generate(model, kv, ctx, prompt, wl.max_new, wl.K)
+        t_e2e = time.perf_counter() - t0
+        alpha = st_a["accepted"] / max(st_a["drafted"], 1)
+        mean_acc = st_a["accepted"] / max(st_a["steps"], 1)
+        step_a, step_g = st_a["ms_decode"] / st_a["steps"], st_g["ms_decode"] / st_g["steps"]
+        rows.append({
+            "workload": f"{name}: the C3 shape with the orbit model, prompt {wl.prompt_len} with corruption {wl.corrupt}, {wl.max_new} new tokens, N={wl.n_max}, K={wl.K}",
+            "tokens_per_s": wl.max_new / t_a, "greedy_tokens_per_s": wl.max_new / t_g, "speedup_vs_greedy": t_g / t_a,
+            "e2e_tokens_per_s": wl.max_new / t_e2e,
+            "decode_speedup_vs_greedy": (st_g["ms_decode"] / st_g["generated"]) / (st_a["ms_decode"] / st_a["generated"]),
+            "hit_ratio_alpha": alpha, "mean_accepted_per_step": mean_acc, "steps": st_a["steps"], "hist_accepted": st_a["hist_accepted"],
+            "bound_alpha_K_plus_1": alpha * wl.K + 1.0,            # the paper's upper bound of the acceleration (Section 4.4)
+            "predicted_decode_speedup": (st_a["generated"] / st_a["steps"]) * step_g / step_a,
+            "ms_per_step_anpd": step_a, "ms_per_step_greedy": step_g, "ms_prefill": st_a["ms_prefill"],
+            "anpd_equals_greedy": bool(np.array_equal(out_a, out_g)), "equals_closed_form": bool(np.array_equal(out_a, want)),
+        })
+    A.anpd_ngram_destroy(ctx)
+    A.anpd_kv_destroy(kv)
+    A.anpd_model_destroy(model)
+    return rows
+
 
 def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
     """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
@@ -287,13 +443,14 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-structured", action="store_true", help="skip the orbit-model runs that follow the C3 line")
     ap.add_argument("--verify-iters", type=int, default=40)
     ap.add_argument("--mode", default="generate", choices=["generate", "verify"],
                     help="verify: the verify-step microbenchmark only (KV length, widths, forced acceptance)")
     ap.add_argument("--kv-len", type=int, nargs="+", default=[2048, 4096])
     ap.add_argument("--widths", type=int, nargs="+", default=[1, 2, 4, 6, 8])
     ap.add_argument("--accept-p", type=float, nargs="+", default=[0.0, 0.5, 0.9])
-    ap.add_argument("--draft-sets", type=int, default=4)
+    ap.add_argument("--draft-sets", type=int, default=32)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -318,7 +475,7 @@ def main() -> None:
     shape = wl.shape
     stream = torch.cuda.Stream()
     t_setup = time.perf_counter()
-    w = make_weights(shape, wl.weight_seed, wl.weights_bf16, device="cuda")
+    w, prompts_all, expected = workload_inputs(wl, device="cuda")
     torch.cuda.synchronize()
     model = A.anpd_model_create(shape, [w[n] for n, _ in tensor_shapes(shape)], stream.cuda_stream)
     want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
@@ -332,13 +489,13 @@ def main() -> None:
     if wl.batch > 1:
         if world > 1:
             raise SystemExit("the batched workload is a single-GPU line")
-        batch_generate_bench(args, A, wl, model, stream, t_setup)
+        batch_generate_bench(args, A, wl, model, stream, t_setup, prompts_all, w_cpu)
         A.anpd_model_destroy(model)
         return
     max_len = wl.prompt_len + wl.max_new + 64
     kv = A.anpd_kv_create(model, max_len)
     ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, stream.cuda_stream)
-    prompt = make_prompts(wl)[0]
+    prompt = prompts_all[0]
     prompt_dev = torch.from_numpy(prompt).cuda()
     out_dev = torch.zeros(wl.max_new, dtype=torch.int32, device="cuda")
     torch.cuda.synchronize()
@@ -428,11 +585,12 @@ def main() -> None:
     gemm_gbs = prof["gemm_bytes"] / (prof["ms_gemm"] * 1e-3) / 1e9 if prof["ms_gemm"] > 0 else 0.0
     roofline = {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections + LM head)",
                 "achieved": gemm_gbs, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                "frac": gemm_gbs / peak, "traffic": NCU_GEMM_TRAFFIC_PER_LAUNCH.get(wl.name),
+                "frac": gemm_gbs / peak, "traffic": gemm_traffic_per_launch(wl),
                 "launches": prof["n_gemm"], "avg_launch_us": prof["ms_gemm"] * 1e3 / max(prof["n_gemm"], 1),
                 "bytes_per_launch": prof["gemm_bytes"] / max(prof["n_gemm"], 1),
-                "step_share": {"gemm_ms": prof["ms_gemm"] / 5, "attn_ms": prof["ms_attn"] / 5,
-                               "other_ms": prof["ms_other"] / 5}}
+                # launched one by one with events around each launch (no graph, no overlap): these add up to more than a step
+                "eager_serialised_ms_per_step": {"gemm": prof["ms_gemm"] / 5, "attention": prof["ms_attn"] / 5,
+                                                 "other": prof["ms_other"] / 5}}
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -460,15 +618,33 @@ def main() -> None:
                         "frac_of_8TBs": verify_gbs / HBM_NOMINAL_GBS, f"frac_of_{peak_kind}_copy": verify_gbs / peak},
         "setup_s": t_setup,
     }
+    # ---- n-gram kernels alone (update + draft of one step), from an event-bracketed (eager) short run ---------------
+    A.anpd_profile_enable(model, True)
+    A.anpd_profile_read(model, True)
+    A.anpd_generate_dev(model, kv, ctx, prompt_dev, min(wl.max_new, 24), wl.K, out_dev)
+    prof_ng = A.anpd_profile_read(model, True)
+    A.anpd_profile_enable(model, False)
+    result["ngram"] = {"step_kernel_us": prof_ng["ms_ngram"] * 1e3 / max(prof_ng["n_ngram"], 1), "launches": prof_ng["n_ngram"],
+                       "note": "update + K chained back-off queries per step (plus the two bulk passes of Initialize), eager launches"}
+    if expected is not None:
+        result["anpd"]["equals_closed_form"] = bool(np.array_equal(anpd_tokens, expected[0][:wl.max_new]))
+
+    # ---- the method at work: same shape and byte traffic, a model whose continuation the drafts can hit -------------
+    if wl.name == "C3" and world == 1 and not args.no_structured:
+        A.anpd_ngram_destroy(ctx)
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(model)
+        ctx = kv = model = None
+        torch.cuda.empty_cache()
+        result["structured_acceptance"] = structured_acceptance(args, A, stream, ("C3-A20", "C3-A60"))
     if want_cpu:
-        big = shape.streamed_params > 3e9
-        sp, sn = (16, 2) if big else ((64, 8) if shape.streamed_params > 1e8 else (wl.prompt_len, wl.max_new))
-        result["cpu_baseline"] = oracle_sample(wl, w_cpu, prompt, sp, sn)
+        result["cpu_baseline"] = oracle_baseline(wl, w_cpu, prompt, st_anpd["accepted"] / max(st_anpd["steps"], 1))
     if rank == 0:
         print(json.dumps(result))
-    A.anpd_ngram_destroy(ctx)
-    A.anpd_kv_destroy(kv)
-    A.anpd_model_destroy(model)
+    if model is not None:
+        A.anpd_ngram_destroy(ctx)
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(model)
     if dist is not None:
         dist.destroy_process_group()
 
