@@ -376,7 +376,6 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&ws.amax_val_rr, (size_t)m->num_sms * ANPD_ROWS * 4}, {(void**)&ws.amax_idx_rr, (size_t)m->num_sms * ANPD_ROWS * 4},
     };
     ws.amax_nblk = ws.amax_blocks;
-    ws.amax_rr = false;
     size_t total = 0;
     for (const Item& it : items) total += up256(it.bytes);
     kv->slab_bytes = total;
@@ -415,6 +414,13 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         if (rc != ANPD_OK) { cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv; return rc; }
     }
 
+    ws.amax_val_use = ws.amax_val;
+    ws.amax_idx_use = ws.amax_idx;
+    {
+        const anpd_status rc = step_kernel_setup(m, kv);
+        if (rc != ANPD_OK) { cudaFree(kv->step_slab); cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv; return rc; }
+    }
+
     // page table: identity, or a fixed permutation of the physical pages
     std::vector<int> pt(kv->total_pages);
     for (int i = 0; i < kv->total_pages; ++i) pt[i] = i;
@@ -445,7 +451,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
     if (!ok) {
         anpd_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__);
-        cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv;
+        cudaFree(kv->step_slab); cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv;
         return ANPD_ERR_CUDA;
     }
     *out = kv;
@@ -455,8 +461,10 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
 anpd_status anpd_kv_destroy(anpd_kv* kv) {
     if (!kv) return ANPD_ERR_ARG;
     cudaStreamSynchronize(kv->m->stream);
+    step_kernel_trace_dump(kv);
     for (auto& g : kv->graphs) cudaGraphExecDestroy(g.second.exec);
     cudaFreeHost(kv->h_seq);
+    cudaFree(kv->step_slab);
     cudaFree(kv->slab);
     delete kv;
     return ANPD_OK;
@@ -516,7 +524,7 @@ static anpd_status read_seqs(anpd_kv* kv) {
     CUDA_TRY(cudaStreamSynchronize(kv->m->stream));
     for (int b = 0; b < kv->batch; ++b) { kv->h_kv_len[b] = kv->h_seq[b].kv_len; kv->h_len_stale[b] = 0; }
     if (*h_err != 0) {
-        std::snprintf(g_last_error, sizeof(g_last_error), "a kernel gave up waiting on a barrier (code %d: 201 GEMM, 202 attention)", *h_err);
+        std::snprintf(g_last_error, sizeof(g_last_error), "a kernel gave up waiting on a barrier (code %d: 201 GEMM, 202 attention, 204 step kernel)", *h_err);
         return ANPD_ERR_CUDA;
     }
     return ANPD_OK;

@@ -868,9 +868,8 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
 anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len) {
     Workspace& ws = kv->ws;
     const int blocks = (mode == ACCEPT_PREFILL) ? 1 : kv->batch;
-    const bool rr = ws.amax_rr;                         // the last forward took the row-range path: its candidates are per CTA
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
-           (launch_k(accept_kernel, blocks, 256, 0, m->stream, kv->seq, rr ? ws.amax_val_rr : ws.amax_val, rr ? ws.amax_idx_rr : ws.amax_idx,
+           (launch_k(accept_kernel, blocks, 256, 0, m->stream, kv->seq, ws.amax_val_use, ws.amax_idx_use,
                      ws.amax_nblk, mode, d_ctxs, seq, last_row, prompt_len)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
@@ -916,16 +915,19 @@ static anpd_status forward_rr_enqueue(anpd_model* m, anpd_kv* kv, int max_pos, b
     lm.logits = want_logits ? ws.logits : nullptr; lm.amax_val = ws.amax_val_rr; lm.amax_idx = ws.amax_idx_rr; lm.V = c.vocab;
     ANPD_TRY(rr_enqueue(RR_LM, m->rr[GK_LM], m->rr_lm, ws.img_h, lm, ws.gemm_err, st, pf));
     ws.amax_nblk = m->rr[GK_LM].G;
-    ws.amax_rr = true;
+    ws.amax_val_use = ws.amax_val_rr;
+    ws.amax_idx_use = ws.amax_idx_rr;
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
 
 anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits) {
     if (m->rr_ready && kv->batch == 1 && rows == ANPD_ROWS && head && !m->plain_gemm) return forward_rr_enqueue(m, kv, max_pos, want_logits);
+    if (kv->step_ready && rows == kv->batch * ANPD_ROWS && head && !m->prof.on) return step_kernel_enqueue(m, kv, max_pos, want_logits);
     const anpd_model_config& c = m->cfg;
     kv->ws.amax_nblk = kv->ws.amax_blocks;
-    kv->ws.amax_rr = false;
+    kv->ws.amax_val_use = kv->ws.amax_val;
+    kv->ws.amax_idx_use = kv->ws.amax_idx;
     Workspace& ws = kv->ws;
     cudaStream_t st = m->stream;
     Profiler* pf = &m->prof;

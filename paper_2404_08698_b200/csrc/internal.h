@@ -295,11 +295,51 @@ struct Workspace {
     float *ss_a, *ss_b;
     float* amax_val_rr; int* amax_idx_rr;
     int amax_nblk;                    // argmax candidates per row left by the last forward (depends on the path it took)
-    bool amax_rr;                     // ... and whether they are in the row-range path's arrays
+    float* amax_val_use; int* amax_idx_use;   // ... and the arrays that hold them
     int* gemm_err;                    // device flag set by a GEMM kernel that gave up waiting
     // TMA views of the activation buffers: [0] decode (batch*8 rows), [1] prefill (PREFILL_ROWS rows)
     CUtensorMap map_h[2][2], map_ao[2][2], map_act[2][2];     // [mode][hi/lo]
     int nb[2];                        // MMA N per mode (rows padded to a multiple of 16)
+};
+
+// Arguments of the persistent step kernel (step_kernel.cu), fixed for a (model, cache) pair.
+struct StepGemm {
+    int N, K, m_tiles, k_blocks, grid;
+    const int* first_cta;             // [m_tiles] CTA that owns a tile's first k-block
+    const int* seg_count;             // [m_tiles] partial sums that cover the tile
+    float* part;                      // [segment][row][ld_part], one buffer per projection kind
+    unsigned long long seg_stride;
+    int ld_part;
+};
+struct StepLayer { const __nv_bfloat16 *wqkv, *wo, *wgu, *wd; const float *attn_norm, *ffn_norm; };
+struct StepParams {
+    alignas(64) CUtensorMap map_k, map_v;
+    StepGemm g[5];
+    const StepLayer* layers;
+    const __nv_bfloat16 *embed, *lm_head;
+    const float* final_norm;
+    int L, d, F, V, Hq, Hkv, hd, dq, rows, stages;
+    float eps, q_scale;
+    const int *row_tok, *row_pos, *row_seq, *row_ok;
+    float* x;
+    // operand images of the projections' inputs (see img_offset in step_kernel.cu): QKV / LM head, gate/up, O, down
+    unsigned char *imgA, *imgB, *img_ao, *img_act;
+    __nv_bfloat16 *q_hi, *q_lo;
+    float *ssA, *ssB;                     // [d / 128][rows] sums of squares of the residual stream per 128-column tile
+    float *pm, *pl, *po;                  // attention page partials
+    float* logits; float* amax_val; int* amax_idx;
+    __nv_bfloat16 *kpool, *vpool;
+    unsigned long long layer_elems;       // elements of one layer of a pool
+    int layer_rows;                       // rows of one layer in the pools' 2-D view
+    const int* page_table; int pages_per_seq;
+    const float *rope_cos, *rope_sin;
+    // phase and arrival counters, zeroed before every step: (L + 1) blocks of `sync_stride` ints
+    int* sync; int sync_stride;
+    int o_dh, o_dqkv, o_dao, o_dhB, o_dact, o_ditems;            // phase counters: finished tiles of the phase that writes hA / q,k,v / ao / hB / act
+    int o_cqkv, o_cattn, o_co, o_cgu, o_cdown, o_clm;   // per-tile arrival counters
+    int* err;
+    unsigned long long* trace;            // optional time stamps (debugging aid), or null
+    int trace_cta;
 };
 
 struct anpd_kv {
@@ -324,8 +364,14 @@ struct anpd_kv {
     // one instantiated CUDA graph per distinct step shape (draft length, mode, attention grid)
     struct StepGraph { cudaGraphExec_t exec; int launches; };
     std::map<uint64_t, StepGraph> graphs;
+    // persistent step kernel: its arguments, the buffers only it uses, and whether decode steps take it
+    StepParams step;
+    bool step_ready;
+    void* step_slab;                  // second gate/up input, per-projection partial sums, tile sums of squares, flags, layer table
+    size_t step_sync_bytes;
+    int step_smem;
     bool use_graphs;
-    bool warm;                        // the first step runs eagerly (one-time function attributes, lazy module loading)
+    bool warm;                       // the first step runs eagerly (one-time function attributes, lazy module loading)
 };
 
 // Forward over `rows` rows (a multiple of 8; 8 consecutive rows always belong to one sequence and
@@ -333,6 +379,13 @@ struct anpd_kv {
 // max_pos: an upper bound of the largest position any row holds (sizes the attention grid).
 // head: also run the LM head and the per-block argmax (false for all but the last prefill pass).
 anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits);
+
+// step_kernel.cu: the whole forward of a decode step as ONE persistent kernel (one CTA per SM).  True if this model / cache
+// pair can take that path (head dimension 128, one query head per kv head, dimensions that are multiples of 128).
+bool step_kernel_eligible(const anpd_model* m, const anpd_kv* kv);
+anpd_status step_kernel_setup(anpd_model* m, anpd_kv* kv);              // fills kv->step (buffers are part of the kv slab)
+anpd_status step_kernel_enqueue(anpd_model* m, anpd_kv* kv, int max_pos, bool want_logits);
+void step_kernel_trace_dump(anpd_kv* kv);
 
 enum AcceptMode { ACCEPT_COMMIT = 0, ACCEPT_PEEK = 1, ACCEPT_PREFILL = 2 };
 anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv);
