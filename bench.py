@@ -425,6 +425,68 @@ def structured_acceptance(args, A, stream, names) -> list:
     return rows
 
 
+def ablation_sweep(args, A, wl, model, stream) -> None:
+    """Draft length K x highest n-gram level N x {multi-level back-off, the level-N table alone} x both query policies on
+    one orbit workload (the paper's Section 4.3 studies K and N on its datasets; its appendix compares N-gram with and
+    without the multi-level back-off).  Every run goes through anpd_generate_dev; the same build's greedy decode is the
+    reference for the speed-up.  Prints one JSON line; a table for reading goes to stderr."""
+    from workloads import orbit_continuation, orbit_permutation, orbit_prompt
+    if wl.orbit_S == 0:
+        raise SystemExit("--mode sweep needs an orbit workload (a random-init model accepts no draft): e.g. --workload C3-A20")
+    pi = orbit_permutation(wl.orbit_S, wl.weight_seed)
+    prompt = orbit_prompt(pi, wl.prompt_len, wl.corrupt, wl.prompt_seed)
+    want = orbit_continuation(pi, prompt[-1], wl.max_new)
+    max_len = wl.prompt_len + wl.max_new + 64
+    kv = A.anpd_kv_create(model, max_len)
+    prompt_dev = torch.from_numpy(prompt).cuda()
+    out_dev = torch.zeros(wl.max_new, dtype=torch.int32, device="cuda")
+
+    def timed(ctx, K: int, reps: int):
+        st = None
+        A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 1e3 / reps, st, out_dev.cpu().numpy().copy()
+
+    ctx0 = A.anpd_ngram_create(2, 2, max_len, 0, stream.cuda_stream)
+    t_greedy, st_g, out_g = timed(ctx0, 0, max(args.steps, 1))
+    A.anpd_ngram_destroy(ctx0)
+    rows, all_equal = [], bool(np.array_equal(out_g, want))
+    for policy in (0, 1):
+        for mln in (True, False):
+            for N in args.sweep_N:
+                ctx = A.anpd_ngram_create(2 if mln else N, N, max_len, policy, stream.cuda_stream)
+                for K in args.sweep_K:
+                    t, st, out = timed(ctx, K, max(args.steps, 1))
+                    all_equal = all_equal and bool(np.array_equal(out, out_g))
+                    alpha = st["accepted"] / max(st["drafted"], 1)
+                    rows.append({"policy": "max-count" if policy == 0 else "last-seen", "levels": f"2..{N}" if mln else f"{N}", "N": N, "K": K,
+                                 "tokens_per_s": wl.max_new / t, "speedup_vs_greedy": t_greedy / t, "steps": st["steps"],
+                                 "drafted": st["drafted"], "accepted": st["accepted"], "hit_ratio_alpha": alpha,
+                                 "mean_accepted_per_step": st["accepted"] / max(st["steps"], 1), "bound_alpha_K_plus_1": alpha * K + 1.0})
+                A.anpd_ngram_destroy(ctx)
+    A.anpd_kv_destroy(kv)
+    print(json.dumps({"metric": "anpd_speedup_sweep", "value": max(r["speedup_vs_greedy"] for r in rows), "unit": "x over greedy (best cell)",
+                      "higher_is_better": True, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"{wl.name}: orbit model at {wl.shape.n_layers}L d{wl.shape.d_model}, prompt {wl.prompt_len} with corruption "
+                                             f"{wl.corrupt}, {wl.max_new} new tokens", "K": args.sweep_K, "N": args.sweep_N,
+                                 "reps": max(args.steps, 1)},
+                      "greedy_tokens_per_s": wl.max_new / t_greedy, "every_stream_equals_greedy_and_closed_form": all_equal, "rows": rows}))
+    for policy in ("max-count", "last-seen"):
+        for levels_kind in ("multi-level (n = 2..N)", "level N alone"):
+            mln = levels_kind.startswith("multi")
+            print(f"\n{wl.name}, policy {policy}, {levels_kind}: speed-up over greedy (hit ratio) by N (rows) and K (columns)", file=sys.stderr)
+            print("  N\\K " + "".join(f"{K:>14d}" for K in args.sweep_K), file=sys.stderr)
+            for N in args.sweep_N:
+                cells = [r for r in rows if r["policy"] == policy and r["N"] == N and (r["levels"].startswith("2..") == mln)]
+                print(f"  {N:>3d} " + "".join(f"  {r['speedup_vs_greedy']:5.2f} ({r['hit_ratio_alpha']:4.2f})" for r in cells), file=sys.stderr)
+
+
 def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
     """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
     time.  `dist` is torch.distributed (or None for one process)."""
@@ -445,8 +507,11 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-structured", action="store_true", help="skip the orbit-model runs that follow the C3 line")
     ap.add_argument("--verify-iters", type=int, default=40)
-    ap.add_argument("--mode", default="generate", choices=["generate", "verify"],
-                    help="verify: the verify-step microbenchmark only (KV length, widths, forced acceptance)")
+    ap.add_argument("--mode", default="generate", choices=["generate", "verify", "sweep"],
+                    help="verify: the verify-step microbenchmark only (KV length, widths, forced acceptance); "
+                         "sweep: K x N x back-off x policy on an orbit workload")
+    ap.add_argument("--sweep-K", type=int, nargs="+", default=[1, 2, 3, 4, 5, 6, 7])
+    ap.add_argument("--sweep-N", type=int, nargs="+", default=[2, 3, 4, 5, 6, 7])
     ap.add_argument("--kv-len", type=int, nargs="+", default=[2048, 4096])
     ap.add_argument("--widths", type=int, nargs="+", default=[1, 2, 4, 6, 8])
     ap.add_argument("--accept-p", type=float, nargs="+", default=[0.0, 0.5, 0.9])
@@ -478,12 +543,16 @@ def main() -> None:
     w, prompts_all, expected = workload_inputs(wl, device="cuda")
     torch.cuda.synchronize()
     model = A.anpd_model_create(shape, [w[n] for n, _ in tensor_shapes(shape)], stream.cuda_stream)
-    want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
+    want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline and args.mode == "generate")
     w_cpu = {k: v.cpu() for k, v in w.items()} if want_cpu else None
     del w
     torch.cuda.empty_cache()
     if args.mode == "verify":
         verify_microbench(args, A, wl, model, stream)
+        A.anpd_model_destroy(model)
+        return
+    if args.mode == "sweep":
+        ablation_sweep(args, A, wl, model, stream)
         A.anpd_model_destroy(model)
         return
     if wl.batch > 1:

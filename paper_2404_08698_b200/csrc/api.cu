@@ -76,6 +76,24 @@ __global__ void greedy_stage_kernel(SeqState* seqs) {
     s.draft_len = 0;
 }
 
+// Last kernel of a step inside the device-resident decoding loop: the loop goes on while a sequence is still active and
+// nothing has failed (a sequence's sticky error, a kernel that gave up waiting, more steps than the caller allowed).
+__global__ void loop_condition_kernel(const SeqState* seqs, int batch, const int* kernel_err, int* steps_left, cudaGraphConditionalHandle handle) {
+    pdl_trigger();
+    pdl_wait();
+    if (threadIdx.x != 0) return;
+    bool go = false;
+    for (int b = 0; b < batch; ++b) {
+        if (seqs[b].error != 0) { go = false; break; }
+        go = go || seqs[b].active != 0;
+    }
+    if (*kernel_err != 0) go = false;
+    const int left = *steps_left - 1;
+    *steps_left = left;
+    if (left <= 0) go = false;
+    cudaGraphSetConditional(handle, go ? 1u : 0u);
+}
+
 inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 uint16_t f32_to_bf16_host(float f) {
@@ -341,6 +359,8 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     kv->total_pages = kv->pages_per_seq * batch;
     kv->staged = false;
     kv->warm = false;
+    kv->loop_ok = std::getenv("ANPD_HOST_LOOP") == nullptr;
+    kv->loop_launches_per_step = 0;
     // the legacy default stream cannot be captured: steps on it are launched one kernel at a time
     kv->use_graphs = std::getenv("ANPD_NO_GRAPH") == nullptr && m->stream != nullptr && m->stream != cudaStreamLegacy;
     kv->h_kv_len.assign(batch, 0);
@@ -369,7 +389,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&ws.attn_m, n_part * 4}, {(void**)&ws.attn_l, n_part * 4}, {(void**)&ws.attn_o, n_part * hd * 4},
         {(void**)&ws.logits, R * V * 4},
         {(void**)&ws.amax_val, R * ws.amax_blocks * 4}, {(void**)&ws.amax_idx, R * ws.amax_blocks * 4},
-        {(void**)&ws.gemm_err, 256},
+        {(void**)&ws.gemm_err, 256}, {(void**)&kv->loop_steps_left, 256},
         {(void**)&ws.img_h, act_img_bytes(c.d_model)}, {(void**)&ws.img_h2, act_img_bytes(c.d_model)},
         {(void**)&ws.img_ao, act_img_bytes(m->dq)}, {(void**)&ws.img_act, act_img_bytes(c.d_ffn)},
         {(void**)&ws.ss_a, (size_t)m->num_sms * ANPD_ROWS * 4}, {(void**)&ws.ss_b, (size_t)m->num_sms * ANPD_ROWS * 4},
@@ -463,6 +483,7 @@ anpd_status anpd_kv_destroy(anpd_kv* kv) {
     cudaStreamSynchronize(kv->m->stream);
     step_kernel_trace_dump(kv);
     for (auto& g : kv->graphs) cudaGraphExecDestroy(g.second.exec);
+    for (auto& g : kv->loop_graphs) cudaGraphExecDestroy(g.second.exec);
     cudaFreeHost(kv->h_seq);
     cudaFree(kv->step_slab);
     cudaFree(kv->slab);
@@ -585,6 +606,79 @@ anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_to
 // (the confirmed token alone); K < 0: the step's inputs were staged by the host.  Then the forward over
 // the batch * 8 rows, argmax / accept and, in COMMIT mode, the KV commit and token-buffer append.
 // Steps of one shape are captured once into a CUDA graph and replayed.
+static anpd_status step_enqueue(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K, int max_pos) {
+    cudaStream_t st = m->stream;
+    if (K > 0) ANPD_TRY(ngram_enqueue_step(d_ctxs, kv->seq, kv->batch, K, st, &m->prof));
+    else if (K == 0) { LAUNCH(&m->prof, st, KC_OTHER, 0, (launch_k(greedy_stage_kernel, kv->batch, 1, 0, st, kv->seq))); }
+    ANPD_TRY(plan_decode_enqueue(m, kv));
+    ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
+    ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
+    return ANPD_OK;
+}
+
+// The whole decoding loop of Algorithm 1 as ONE graph launch: a conditional WHILE node whose body is the step (update +
+// draft, row plan, forward, accept / commit) followed by a kernel that decides whether another step runs.  The host neither
+// launches nor synchronises per step.  The body's attention grid is sized for the longest context the run can reach
+// (`max_pos_bound`); pages beyond a sequence's current length are skipped inside the kernels.  Returns ANPD_ERR_STATE if
+// the loop cannot be built on this stream / driver (the caller then steps from the host).
+static anpd_status decode_loop_enqueue(anpd_model* m, anpd_kv* kv, const NgramDev* d_ctxs, int K, int max_pos_bound, int max_steps) {
+    if (!kv->use_graphs || m->prof.on || !kv->loop_ok) return ANPD_ERR_STATE;
+    cudaStream_t st = m->stream;
+    const uint64_t key = (uint64_t)(max_pos_bound / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)(d_ctxs ? 1 : 0) << 29);
+    auto it = kv->loop_graphs.find(key);
+    if (it == kv->loop_graphs.end()) {
+        if (!kv->warm) {                                // one eager step first: function attributes, lazy module loading
+            kv->warm = true;
+            return ANPD_ERR_STATE;
+        }
+        cudaGraph_t graph = nullptr;
+        cudaGraphExec_t exec = nullptr;
+        bool ok = cudaGraphCreate(&graph, 0) == cudaSuccess;
+        cudaGraphConditionalHandle handle = 0;
+        ok = ok && cudaGraphConditionalHandleCreate(&handle, graph, 1, cudaGraphCondAssignDefault) == cudaSuccess;
+        cudaGraphNodeParams np = {};
+        np.type = cudaGraphNodeTypeConditional;
+        np.conditional.handle = handle;
+        np.conditional.type = cudaGraphCondTypeWhile;
+        np.conditional.size = 1;
+        cudaGraphNode_t node = nullptr;
+        ok = ok && cudaGraphAddNode(&node, graph, nullptr, 0, &np) == cudaSuccess;
+        int launches = 0;
+        if (ok) {
+            cudaGraph_t body = np.conditional.phGraph_out[0];
+            const long long before = g_launch_count.load();
+            ok = cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+            if (ok) {
+                anpd_status rc = step_enqueue(m, kv, ACCEPT_COMMIT, false, d_ctxs, K, max_pos_bound);
+                if (rc == ANPD_OK) {
+                    LAUNCH(&m->prof, st, KC_OTHER, 0,
+                           (launch_k(loop_condition_kernel, 1, 32, 0, st, kv->seq, kv->batch, kv->ws.gemm_err, kv->loop_steps_left, handle)));
+                    if (cudaGetLastError() != cudaSuccess) rc = ANPD_ERR_CUDA;
+                }
+                cudaGraph_t captured = nullptr;
+                const cudaError_t ce = cudaStreamEndCapture(st, &captured);
+                ok = rc == ANPD_OK && ce == cudaSuccess;
+            }
+            launches = (int)(g_launch_count.load() - before);
+            g_launch_count.fetch_sub(launches);         // capturing runs nothing
+        }
+        ok = ok && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess;
+        if (graph) cudaGraphDestroy(graph);
+        if (!ok) {
+            cudaGetLastError();
+            if (exec) cudaGraphExecDestroy(exec);
+            kv->loop_ok = false;                        // step from the host for good
+            return ANPD_ERR_STATE;
+        }
+        it = kv->loop_graphs.emplace(key, anpd_kv::StepGraph{exec, launches}).first;
+    }
+    CUDA_TRY(cudaMemcpyAsync(kv->loop_steps_left, &max_steps, sizeof(int), cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaGraphLaunch(it->second.exec, st));
+    std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1);
+    kv->loop_launches_per_step = it->second.launches;
+    return ANPD_OK;
+}
+
 static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K = -1) {
     ANPD_TRY(check_device(m));
     int max_pos = 0;
@@ -595,14 +689,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
         max_pos = std::max(max_pos, kv->h_kv_len[b] + ANPD_ROWS - 1);
     }
     cudaStream_t st = m->stream;
-    auto enqueue = [&]() -> anpd_status {
-        if (K > 0) ANPD_TRY(ngram_enqueue_step(d_ctxs, kv->seq, kv->batch, K, st, &m->prof));
-        else if (K == 0) { LAUNCH(&m->prof, st, KC_OTHER, 0, (launch_k(greedy_stage_kernel, kv->batch, 1, 0, st, kv->seq))); }
-        ANPD_TRY(plan_decode_enqueue(m, kv));
-        ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
-        ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
-        return ANPD_OK;
-    };
+    auto enqueue = [&]() -> anpd_status { return step_enqueue(m, kv, mode, want_logits, d_ctxs, K, max_pos); };
     if (m->prof.on || !kv->use_graphs || !kv->warm) {
         kv->warm = true;
         NoPdlScope no_overlap(m->prof.on);            // per-launch timing needs kernels that do not overlap
@@ -739,13 +826,24 @@ static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* 
         for (int b = 0; b < B; ++b) ANPD_TRY(seq_error_status(kv->h_seq[b]));
         bool any_active = true;
         while (any_active) {
-            ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs, K));
+            // the device-resident loop runs every remaining step in one launch; where it is not available (first step of a
+            // handle, legacy stream, profiling, a driver that refuses the graph) the host steps and reads the state back
+            const int max_pos_bound = std::min(prompt_len + max_new + 2 * ANPD_ROWS, kv->max_len) - 1;
+            const anpd_status lrc = decode_loop_enqueue(m, kv, kv->d_ctxs, K, max_pos_bound, max_new + 2);
+            if (lrc == ANPD_OK) g_launch_count += 0;    // counted below from the steps the sequences report
+            else if (lrc != ANPD_ERR_STATE) return lrc;
+            else ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs, K));
+            int steps_before = 0;
+            for (int b = 0; b < B; ++b) steps_before = std::max(steps_before, kv->h_seq[b].steps);
             ANPD_TRY(read_seqs(kv));
             any_active = false;
+            int steps_after = 0;
             for (int b = 0; b < B; ++b) {
                 ANPD_TRY(seq_error_status(kv->h_seq[b]));
                 any_active = any_active || kv->h_seq[b].active;
+                steps_after = std::max(steps_after, kv->h_seq[b].steps);
             }
+            if (lrc == ANPD_OK) g_launch_count += (long long)kv->loop_launches_per_step * std::max(steps_after - steps_before, 1);
         }
         CUDA_TRY(cudaEventRecord(e2, st));
         CUDA_TRY(cudaEventSynchronize(e2));

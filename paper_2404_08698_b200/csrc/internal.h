@@ -364,6 +364,11 @@ struct anpd_kv {
     // one instantiated CUDA graph per distinct step shape (draft length, mode, attention grid)
     struct StepGraph { cudaGraphExec_t exec; int launches; };
     std::map<uint64_t, StepGraph> graphs;
+    // the device-resident decoding loop: one graph (a WHILE node around the step) per (draft length, context bound)
+    std::map<uint64_t, StepGraph> loop_graphs;
+    bool loop_ok;                     // false once building such a graph has failed, or when ANPD_HOST_LOOP is set
+    int* loop_steps_left;             // device: steps the running loop may still take
+    int loop_launches_per_step;
     // persistent step kernel: its arguments, the buffers only it uses, and whether decode steps take it
     StepParams step;
     bool step_ready;

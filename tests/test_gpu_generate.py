@@ -237,3 +237,41 @@ def test_generate_error_paths(A, c1):
         assert e.value.status == A.ERR_RANGE
     finally:
         A.anpd_ngram_destroy(ctx)
+
+
+def test_device_resident_loop_equals_host_stepped_loop(A, monkeypatch):
+    """The decoding loop as one graph launch (a WHILE node around the step, no host round trip per step) against the
+    same loop stepped from the host (ANPD_HOST_LOOP=1): same tokens, same statistics, for ANPD and for greedy, on a
+    model that accepts drafts (orbit workload) and on the random tiny model; the device loop launches the same kernels
+    per step plus the one that decides whether to go on."""
+    from workloads import workload_inputs
+    results = {}
+    for host_loop in (False, True):
+        if host_loop:
+            monkeypatch.setenv("ANPD_HOST_LOOP", "1")
+        for name in ("C1-A50", "C1"):
+            wl = WORKLOADS[name]
+            w, prompts, _ = workload_inputs(wl)
+            st = new_stream()
+            m = gpu_model(A, wl.shape, w, st)
+            kv = A.anpd_kv_create(m, 512)
+            ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, 512, 0, st)
+            try:
+                A.anpd_generate(m, kv, ctx, prompts[0], 8, wl.K)                  # first run of a handle: eager first step
+                A.anpd_launch_count(True)
+                out, stats = A.anpd_generate(m, kv, ctx, prompts[0], wl.max_new, wl.K)
+                launches = A.anpd_launch_count(True)
+                greedy, gstats = A.anpd_generate(m, kv, ctx, prompts[0], wl.max_new, 0)
+            finally:
+                A.anpd_ngram_destroy(ctx)
+                A.anpd_kv_destroy(kv)
+                A.anpd_model_destroy(m)
+            keep = {k: stats[k] for k in ("steps", "drafted", "accepted", "generated", "hist_accepted")}
+            results[(name, host_loop)] = (out.tolist(), greedy.tolist(), keep, gstats["steps"], launches)
+    for name in ("C1-A50", "C1"):
+        dev, host = results[(name, False)], results[(name, True)]
+        assert dev[:4] == host[:4], name
+        assert dev[0] == dev[1]                                                  # losslessness in the device loop
+        steps = dev[2]["steps"]
+        assert dev[4] - host[4] == steps, (dev[4], host[4], steps)               # one more kernel per step, nothing else
+    assert results[("C1-A50", False)][2]["accepted"] > 0
