@@ -156,7 +156,7 @@ static anpd_status model_make_plans(anpd_model* m) {
         max_tiles = std::max(max_tiles, m->plan[k].m_tiles);
         m->max_segs = std::max(m->max_segs, m->plan[k].max_segs);
     }
-    ints += max_tiles;
+    ints += 4 * (size_t)max_tiles;
     std::vector<int> host(ints);
     CUDA_TRY(cudaMalloc((void**)&m->d_plan_tables, ints * sizeof(int)));
     size_t off = 0;
@@ -169,6 +169,11 @@ static anpd_status model_make_plans(anpd_model* m) {
     }
     m->d_ones = m->d_plan_tables + off;
     for (int i = 0; i < max_tiles; ++i) host[off + i] = 1;
+    m->d_const_segs[0] = m->d_const_segs[1] = m->d_ones;
+    for (int k = 2; k <= 3; ++k) {
+        m->d_const_segs[k] = m->d_plan_tables + off + (size_t)(k - 1) * max_tiles;
+        for (int i = 0; i < max_tiles; ++i) host[off + (size_t)(k - 1) * max_tiles + i] = k;
+    }
     CUDA_TRY(cudaMemcpy(m->d_plan_tables, host.data(), ints * sizeof(int), cudaMemcpyHostToDevice));
     return ANPD_OK;
 }
@@ -366,7 +371,8 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     kv->h_kv_len.assign(batch, 0);
     kv->h_len_stale.assign(batch, 0);
     Workspace& ws = kv->ws;
-    ws.r_max = std::max(PREFILL_ROWS, batch * ANPD_ROWS);
+    ws.prefill_rows = std::min(PREFILL_ROWS_MAX, (kv->max_len + 255) / 256 * 256);
+    ws.r_max = std::max(ws.prefill_rows, batch * ANPD_ROWS);
     ws.n_max_out = (std::max(std::max(m->nqkv, 2 * c.d_ffn), std::max(c.d_model, c.vocab)) + 127) / 128 * 128;
     ws.splits_max = m->max_segs;
     ws.amax_blocks = (c.vocab + 1023) / 1024;
@@ -384,10 +390,11 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&ws.x, R * d * 4}, {(void**)&ws.h_hi, R * d * 2}, {(void**)&ws.h_lo, R * d * 2},
         {(void**)&ws.ao_hi, R * m->dq * 2}, {(void**)&ws.ao_lo, R * m->dq * 2},
         {(void**)&ws.act_hi, R * F * 2}, {(void**)&ws.act_lo, R * F * 2},
-        {(void**)&ws.part, (size_t)ws.splits_max * R * ws.n_max_out * 4},
+        // decode steps leave up to splits_max partial sums per output, prompt passes up to three (their cut along K)
+        {(void**)&ws.part, std::max((size_t)ws.splits_max * batch * ANPD_ROWS, 3 * R) * ws.n_max_out * 4},
         {(void**)&ws.q_hi, R * m->dq * 2}, {(void**)&ws.q_lo, R * m->dq * 2},
         {(void**)&ws.attn_m, n_part * 4}, {(void**)&ws.attn_l, n_part * 4}, {(void**)&ws.attn_o, n_part * hd * 4},
-        {(void**)&ws.logits, R * V * 4},
+        {(void**)&ws.logits, (size_t)batch * ANPD_ROWS * V * 4},
         {(void**)&ws.amax_val, R * ws.amax_blocks * 4}, {(void**)&ws.amax_idx, R * ws.amax_blocks * 4},
         {(void**)&ws.gemm_err, 256}, {(void**)&kv->loop_steps_left, 256},
         {(void**)&ws.img_h, act_img_bytes(c.d_model)}, {(void**)&ws.img_h2, act_img_bytes(c.d_model)},
@@ -408,10 +415,10 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
 
     // TMA views of the GEMM inputs: decode rows (batch * 8) and prefill rows, each padded to the MMA's N
     {
-        const int mode_rows[2] = {batch * ANPD_ROWS, PREFILL_ROWS};
+        const int mode_rows[2] = {batch * ANPD_ROWS, ws.prefill_rows};
         anpd_status rc = ANPD_OK;
         for (int md = 0; md < 2 && rc == ANPD_OK; ++md) {
-            const int rows = mode_rows[md], nb = (rows + 15) / 16 * 16;
+            const int rows = mode_rows[md], nb = md == 0 ? (rows + 15) / 16 * 16 : 128;
             ws.nb[md] = nb;
             struct { CUtensorMap* maps; const bf16* hi; const bf16* lo; int K; } bufs[3] = {
                 {ws.map_h[md], ws.h_hi, ws.h_lo, c.d_model}, {ws.map_ao[md], ws.ao_hi, ws.ao_lo, m->dq}, {ws.map_act[md], ws.act_hi, ws.act_lo, c.d_ffn}};
@@ -527,13 +534,17 @@ static anpd_status kv_reset(anpd_kv* kv, const int* stop_at) {
 static anpd_status prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, const int32_t* prompt, int prompt_len,
                                    const NgramDev* d_ctxs) {
     CUDA_TRY(cudaMemcpyAsync(kv->d_prompt, prompt, sizeof(int) * (size_t)prompt_len, cudaMemcpyDefault, m->stream));
-    for (int start = 0; start < prompt_len; start += PREFILL_ROWS) {
-        const int n = std::min(PREFILL_ROWS, prompt_len - start);
+    const int pass_rows = kv->ws.prefill_rows;
+    for (int start = 0; start < prompt_len; start += pass_rows) {
+        const int n = std::min(pass_rows, prompt_len - start);
         const int rows = (n + ANPD_ROWS - 1) / ANPD_ROWS * ANPD_ROWS;
         const bool last = start + n >= prompt_len;
-        ANPD_TRY(plan_prefill_enqueue(m, kv, seq, start, prompt_len, rows));
-        ANPD_TRY(forward_enqueue(m, kv, rows, std::min(start + rows - 1, kv->max_len - 1), last, false));
-        if (last) ANPD_TRY(accept_enqueue(m, kv, ACCEPT_PREFILL, d_ctxs, seq, prompt_len - 1 - start, prompt_len));
+        // the row plan also covers the padding up to a multiple of 64 rows: the prompt attention takes up to 64 rows per item
+        ANPD_TRY(plan_prefill_enqueue(m, kv, seq, start, prompt_len, std::min((rows + 63) / 64 * 64, kv->ws.r_max)));
+        const int last_row = prompt_len - 1 - start;
+        ANPD_TRY(forward_enqueue(m, kv, rows, std::min(start + rows - 1, kv->max_len - 1), last, false, last_row));
+        // the LM head of a prompt pass runs on the last token's group of 8 rows, moved to rows 0-7
+        if (last) ANPD_TRY(accept_enqueue(m, kv, ACCEPT_PREFILL, d_ctxs, seq, rows == kv->batch * ANPD_ROWS ? last_row : last_row % ANPD_ROWS, prompt_len));
     }
     return ANPD_OK;
 }

@@ -31,6 +31,7 @@
 #include <math_constants.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 typedef __nv_bfloat16 bf16;
 
@@ -69,7 +70,10 @@ __device__ __forceinline__ void slot_bar(int slot) { asm volatile("bar.sync %0, 
 
 struct AttnItem { int c, kvh, r0, pos_lo, seq; };
 
-template <int G, int S>
+// PF (prompt passes of a model with one query head per kv head): an item's 8 x G query vectors are 8 x G consecutive rows of ONE
+// head (consecutive positions of the prompt) instead of 8 rows of G heads, so a page is fetched once for 8 x G rows; AttnItem::kvh
+// then holds the head.
+template <int G, int S, bool PF>
 __global__ void __launch_bounds__(AttnCfg<G, S>::THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const bf16* __restrict__ q_hi,
                const bf16* __restrict__ q_lo, const int* __restrict__ page_table, int pages_per_seq, const int* __restrict__ row_pos,
@@ -117,12 +121,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int stride = gridDim.x * SLOTS;
     auto decode = [&](int it, AttnItem& out) {
         const int rest = it / chunks;
-        out.c = it % chunks; out.kvh = rest % Hkv; out.r0 = (rest / Hkv) * ANPD_ROWS;
+        out.c = it % chunks; out.kvh = rest % Hkv; out.r0 = (rest / Hkv) * (PF ? Q : ANPD_ROWS);
     };
     auto next_item = [&](int it, AttnItem& out) -> int {
         for (; it < n_items; it += stride) {
             decode(it, out);
-            const int hi = row_pos[out.r0 + ANPD_ROWS - 1];          // three independent loads
+            const int hi = row_pos[out.r0 + (PF ? Q : ANPD_ROWS) - 1];   // three independent loads
             out.pos_lo = row_pos[out.r0];
             out.seq = row_seq[out.r0];
             if (out.c * KV_PAGE <= hi) return it;
@@ -147,7 +151,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             if (idx < N * 16) {
                 const int n = idx >> 4, c16 = idx & 15;
                 const int qn = n % Q, g = qn >> 3, r = qn & 7;
-                const bf16* src = (n < Q ? q_hi : q_lo) + (size_t)(a.r0 + r) * Hq * HD + (size_t)(a.kvh * G + g) * HD + c16 * 8;
+                const bf16* src = (n < Q ? q_hi : q_lo) + (PF ? (size_t)(a.r0 + qn) * Hq * HD + (size_t)a.kvh * HD
+                                                              : (size_t)(a.r0 + r) * Hq * HD + (size_t)(a.kvh * G + g) * HD) + c16 * 8;
                 regs[u] = *(const uint4*)src;
             }
         }
@@ -214,7 +219,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const int key = cur.c * KV_PAGE + t;
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
-            if (key > cur.pos_lo + (q & 7)) s[q] = -CUDART_INF_F;
+            if (key > cur.pos_lo + (PF ? q : (q & 7))) s[q] = -CUDART_INF_F;
             float mx = s[q];
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if (lane == 0) red_max[slot][warp][q] = mx;
@@ -252,7 +257,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             }
         }
         if (t < Q) {
-            const size_t out = ((size_t)(cur.r0 + (t & 7)) * Hq + (cur.kvh * G + (t >> 3))) * pages_per_seq + cur.c;
+            const size_t out = (PF ? (size_t)(cur.r0 + t) * Hq + cur.kvh : (size_t)(cur.r0 + (t & 7)) * Hq + (cur.kvh * G + (t >> 3))) * pages_per_seq + cur.c;
             float mt = m[0];
 #pragma unroll
             for (int q = 1; q < Q; ++q) mt = (q == t) ? m[q] : mt;
@@ -268,7 +273,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             for (int c0 = 0; c0 < N; c0 += 16) tc_ld16(lane_base + (uint32_t)c0, v + c0);
 #pragma unroll
             for (int q = 0; q < Q; ++q) {
-                const size_t out = ((size_t)(cur.r0 + (q & 7)) * Hq + (cur.kvh * G + (q >> 3))) * pages_per_seq + cur.c;
+                const size_t out = (PF ? (size_t)(cur.r0 + q) * Hq + cur.kvh : (size_t)(cur.r0 + (q & 7)) * Hq + (cur.kvh * G + (q >> 3))) * pages_per_seq + cur.c;
                 po[out * HD + t] = v[q] + v[Q + q];
             }
         }
@@ -292,29 +297,255 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     }
 }
 
-template <int G, int S>
+// ---------------------------------------------------------------------------------------------
+// Prompt passes (one query head per kv head): causal attention of a tile of 16 consecutive rows of one head over all the
+// pages those rows may see, page after page with a running maximum, so that no per-page partial leaves the SM and no merge
+// kernel follows.  Products, operand layouts and the page buffer's K -> V^T -> next K rotation are those of the kernel
+// above.  Per page: S^T = K . Q^T; the page's maxima raise the running maxima m; P = 2^(S - m) (hi + lo) goes to shared
+// memory; thread t keeps the sum of its own key's weights, rescaled by 2^(m_old - m) like the output accumulator
+// O[q] (thread = output dimension, in registers), to which O^T = V^T . P^T of the page is added.  The weights' sums are
+// reduced across threads once, at the end.  Pages are visited in ascending order: the result depends on the row's own
+// position and inputs only.
+// ---------------------------------------------------------------------------------------------
+constexpr int PFQ = 16, PFN = 32;            // rows per tile; MMA N (hi + lo terms)
+constexpr int PF_SLOTS = 4;
+constexpr int PF_B_BYTES = PFN * 256;
+constexpr int PF_SLOT_BYTES = 2 * PAGE_ATOM + 2 * PF_B_BYTES;
+constexpr size_t PF_SMEM = (size_t)PF_SLOTS * PF_SLOT_BYTES + 1024;
+
+__global__ void __launch_bounds__(PF_SLOTS * 128, 1)
+attn_prompt_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const bf16* __restrict__ q_hi,
+                   const bf16* __restrict__ q_lo, const int* __restrict__ page_table, int pages_per_seq, const int* __restrict__ row_pos,
+                   const int* __restrict__ row_seq, int H, int layer_row0, int n_tiles, bf16* __restrict__ ao_hi, bf16* __restrict__ ao_lo,
+                   int* err) {
+    extern __shared__ __align__(1024) unsigned char attn_tc_smem[];
+    __shared__ uint64_t bar_k[PF_SLOTS], bar_v[PF_SLOTS], bar_s[PF_SLOTS], bar_o[PF_SLOTS];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ float red_max[PF_SLOTS][4][PFQ];
+    __shared__ float red_sum[PF_SLOTS][4][PFQ];
+
+    pdl_trigger();
+    const int slot = threadIdx.x >> 7, t = threadIdx.x & 127, warp = t >> 5, lane = t & 31;
+    unsigned char* smem = attn_tc_smem + ((1024u - (smem_u32(attn_tc_smem) & 1023u)) & 1023u) + (size_t)slot * PF_SLOT_BYTES;
+    unsigned char* Bs = smem;
+    unsigned char* Qs = smem + 2 * PAGE_ATOM;
+    unsigned char* Ps = Qs + PF_B_BYTES;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < PF_SLOTS; ++i) { mbar_init(&bar_k[i], 1); mbar_init(&bar_v[i], 1); mbar_init(&bar_s[i], 1); mbar_init(&bar_o[i], 1); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(128u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *((volatile uint32_t*)&tmem_slot) + (uint32_t)(slot * PFN);
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    volatile int* abortp = &abort_flag;
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(PFN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    const uint64_t pol = policy_evict_last();           // a page is read by every row tile behind it
+
+    pdl_wait();
+
+    auto load_page = [&](const CUtensorMap* map, uint64_t* bar, int seq, int c, int h) {
+        const int row = layer_row0 + (page_table[seq * pages_per_seq + c] * H + h) * KV_PAGE;
+        mbar_expect_tx(bar, 2 * PAGE_ATOM);
+        tma_load_2d(Bs, map, 0, row, bar, pol);
+        tma_load_2d(Bs + PAGE_ATOM, map, 64, row, bar, pol);
+    };
+    uint32_t n_k = 0, n_v = 0, n_s = 0, n_o = 0;        // completed uses of the slot's four barriers (their parities)
+    uint32_t k_issued = 0, v_issued = 0;
+    bool ok = true;
+    // tile -> (head, 16 rows); tiles with the most pages first (they are the longest)
+    for (int it = slot * gridDim.x + blockIdx.x; it < n_tiles * H && ok; it += gridDim.x * PF_SLOTS) {
+        const int rt = n_tiles - 1 - it / H, h = it % H;
+        const int r0 = rt * PFQ;
+        const int pos_lo = row_pos[r0], pos_hi = row_pos[r0 + PFQ - 1], seq = row_seq[r0];
+        const int n_pages = pos_hi / KV_PAGE + 1;
+        if (t == 0) { load_page(&map_k, &bar_k[slot], seq, 0, h); ++k_issued; }
+        // queries: operand row n is row n % 16 of the tile (hi term for n < 16, lo term after); 16-byte chunks
+#pragma unroll
+        for (int u = 0; u < (PFN * 16) / 128; ++u) {
+            const int idx = t + u * 128, n = idx >> 4, c16 = idx & 15;
+            const bf16* src = (n < PFQ ? q_hi : q_lo) + (size_t)(r0 + (n % PFQ)) * H * HD + (size_t)h * HD + c16 * 8;
+            *(uint4*)(Qs + b_operand_offset<PFN>(n, c16 * 8)) = *(const uint4*)src;
+        }
+        fence_async_smem();
+        slot_bar(slot);
+        float m_run[PFQ], l_thr[PFQ], o_acc[PFQ];
+#pragma unroll
+        for (int q = 0; q < PFQ; ++q) { m_run[q] = -CUDART_INF_F; l_thr[q] = 0.0f; o_acc[q] = 0.0f; }
+        for (int c = 0; c < n_pages && ok; ++c) {
+            // ---- S^T = K . Q^T ----
+            if (t == 0) {
+                if (mbar_wait(&bar_k[slot], n_k & 1u, abortp)) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int k16 = 0; k16 < HD / 16; ++k16) {
+                        const uint64_t adv = (uint64_t)((k16 & 3) * 2);
+                        tc_mma_bf16(tmem_base, make_smem_desc(smem_u32(Bs + (k16 >> 2) * PAGE_ATOM)) + adv,
+                                    make_smem_desc(smem_u32(Qs + (k16 >> 2) * (PFN * 128))) + adv, idesc, k16 > 0 ? 1u : 0u);
+                    }
+                    tc_commit(&bar_s[slot]);
+                }
+            }
+            ++n_k;
+            ok = mbar_wait(&bar_s[slot], n_s & 1u, abortp);
+            ++n_s;
+            if (!ok) break;
+            tc_fence_after();
+            if (t == 0) { load_page(&map_v, &bar_v[slot], seq, c, h); ++v_issued; }     // the first product is done with the page buffer
+            float s[PFQ];
+            {
+                float v[PFN];
+                tc_ld16(lane_base, v);
+                tc_ld16(lane_base + 16u, v + 16);
+#pragma unroll
+                for (int q = 0; q < PFQ; ++q) s[q] = v[q] + v[PFQ + q];
+            }
+            const int key = c * KV_PAGE + t;
+#pragma unroll
+            for (int q = 0; q < PFQ; ++q) {
+                if (key > pos_lo + q) s[q] = -CUDART_INF_F;
+                float mx = s[q];
+                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                if (lane == 0) red_max[slot][warp][q] = mx;
+            }
+            tc_fence_before();
+            slot_bar(slot);
+            float scale[PFQ];
+#pragma unroll
+            for (int q = 0; q < PFQ; ++q) {
+                const float mp = fmaxf(fmaxf(red_max[slot][0][q], red_max[slot][1][q]), fmaxf(red_max[slot][2][q], red_max[slot][3][q]));
+                const float m_new = fmaxf(m_run[q], mp);
+                const bool none = (m_new == -CUDART_INF_F);
+                scale[q] = (none || m_run[q] == -CUDART_INF_F) ? 0.0f : exp2f(m_run[q] - m_new);
+                const float pw = none ? 0.0f : exp2f(s[q] - m_new);
+                const bf16 hh = __float2bfloat16_rn(pw);
+                const bf16 ll = __float2bfloat16_rn(pw - __bfloat162float(hh));
+                *(bf16*)(Ps + b_operand_offset<PFN>(q, t)) = hh;
+                *(bf16*)(Ps + b_operand_offset<PFN>(PFQ + q, t)) = ll;
+                l_thr[q] = fmaf(l_thr[q], scale[q], pw);
+                m_run[q] = m_new;
+            }
+            fence_async_smem();
+            slot_bar(slot);
+            // ---- O^T = V^T . P^T ----
+            if (t == 0) {
+                if (mbar_wait(&bar_v[slot], n_v & 1u, abortp)) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int k16 = 0; k16 < KV_PAGE / 16; ++k16) {
+                        const uint64_t adv = (uint64_t)((k16 & 3) * 2);
+                        tc_mma_bf16(tmem_base, make_smem_desc(smem_u32(Bs + (k16 >> 2) * PAGE_ATOM)) + adv,
+                                    make_smem_desc(smem_u32(Ps + (k16 >> 2) * (PFN * 128))) + adv, idesc, k16 > 0 ? 1u : 0u);
+                    }
+                    tc_commit(&bar_o[slot]);
+                }
+            }
+            ++n_v;
+            ok = mbar_wait(&bar_o[slot], n_o & 1u, abortp);
+            ++n_o;
+            if (!ok) break;
+            tc_fence_after();
+            if (c + 1 < n_pages && t == 0) { load_page(&map_k, &bar_k[slot], seq, c + 1, h); ++k_issued; }   // the second product is done with the buffer
+            {
+                float v[PFN];
+                tc_ld16(lane_base, v);
+                tc_ld16(lane_base + 16u, v + 16);
+#pragma unroll
+                for (int q = 0; q < PFQ; ++q) o_acc[q] = fmaf(o_acc[q], scale[q], v[q] + v[PFQ + q]);
+            }
+            tc_fence_before();
+            slot_bar(slot);                              // the next first product overwrites the columns just read
+        }
+        if (!ok) break;
+        // the weights' sums over all keys: within a warp, then the four warps in order
+#pragma unroll
+        for (int q = 0; q < PFQ; ++q) {
+            float sum = l_thr[q];
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0) red_sum[slot][warp][q] = sum;
+        }
+        slot_bar(slot);
+#pragma unroll
+        for (int q = 0; q < PFQ; ++q) {
+            const float L = (red_sum[slot][0][q] + red_sum[slot][1][q]) + (red_sum[slot][2][q] + red_sum[slot][3][q]);
+            const float o = o_acc[q] / L;
+            const bf16 hh = __float2bfloat16_rn(o);
+            const bf16 ll = __float2bfloat16_rn(o - __bfloat162float(hh));
+            const size_t out = (size_t)(r0 + q) * H * HD + (size_t)h * HD + t;
+            ao_hi[out] = hh;
+            ao_lo[out] = ll;
+        }
+        slot_bar(slot);                                  // the staging buffers and the reduction scratch are free again
+    }
+    if (t == 0 && abort_flag) {
+        if (k_issued) for (unsigned spin = 0; spin < WAIT_LIMIT && !mbar_try_wait(&bar_k[slot], (k_issued - 1) & 1u); ++spin) {}
+        if (v_issued) for (unsigned spin = 0; spin < WAIT_LIMIT && !mbar_try_wait(&bar_v[slot], (v_issued - 1) & 1u); ++spin) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(err, ATTN_ERR_TIMEOUT);
+    if (threadIdx.x < 32) {
+        tc_fence_after();
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*((volatile uint32_t*)&tmem_slot)), "r"(128u) : "memory");
+    }
+}
+
+template <int G, int S, bool PF = false>
 anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int chunks) {
     typedef AttnCfg<G, S> Cfg;
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
     static bool attr_set[64] = {false};
     if (first_call_on_device(attr_set)) {
-        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G, S, PF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
     }
     const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
-    const int n_items = chunks * c.n_kv_heads * (rows / ANPD_ROWS);
+    const int n_items = PF ? chunks * c.n_q_heads * ((rows + Cfg::Q - 1) / Cfg::Q) : chunks * c.n_kv_heads * (rows / ANPD_ROWS);
     const int grid = std::min(m->num_sms, n_items);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_tc_kernel<G, S>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
-                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
+           (launch_k(attn_tc_kernel<G, S, PF>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
+                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, PF ? c.n_q_heads : c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
                      ws.attn_l, ws.attn_o, ws.gemm_err)));
     return ANPD_OK;
 }
 
 }  // namespace
 
-anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos) {
+// Attention of a prompt pass, straight to the O projection's input (no page partials, no merge).  rows: a multiple of 8; the
+// row plan must cover the padding up to a multiple of 16.
+anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows) {
+    const anpd_model_config& c = m->cfg;
+    Workspace& ws = kv->ws;
+    static bool attr_set[64] = {false};
+    if (first_call_on_device(attr_set)) {
+        CUDA_TRY(cudaFuncSetAttribute(attn_prompt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PF_SMEM));
+    }
+    const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
+    const int n_tiles = (rows + PFQ - 1) / PFQ;
+    const int grid = std::min(m->num_sms, (n_tiles * c.n_q_heads + PF_SLOTS - 1) / PF_SLOTS);
+    LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
+           (launch_k(attn_prompt_kernel, grid, PF_SLOTS * 128, PF_SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
+                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, layer_row0, n_tiles, ws.ao_hi, ws.ao_lo, ws.gemm_err)));
+    CUDA_TRY(cudaGetLastError());
+    return ANPD_OK;
+}
+
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool prompt_pass) {
     const int chunks = max_pos / KV_PAGE + 1;
+    if (prompt_pass && m->cfg.n_q_heads == m->cfg.n_kv_heads) {
+        // rows are consecutive positions of one sequence: 16 of them share every page fetch (32 or 64 rows per item measured slower)
+        return launch_attn_tc<2, 4, true>(m, kv, layer, rows, chunks);
+    }
     const int n_items = chunks * m->cfg.n_kv_heads * (rows / ANPD_ROWS);
     switch (m->cfg.n_q_heads / m->cfg.n_kv_heads) {
         // one query head per kv head fits five slots; while every item finds a slot with four, four are faster

@@ -784,6 +784,18 @@ __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict_
     }
 }
 
+// rows [from, from + 8) of the normalised activations -> rows [0, 8)
+__global__ void move_rows_kernel(bf16* __restrict__ h_hi, bf16* __restrict__ h_lo, int from, int d) {
+    pdl_trigger();
+    pdl_wait();
+    if (from == 0) return;
+    const int r = blockIdx.x;
+    for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+        ((uint4*)(h_hi + (size_t)r * d))[i] = ((const uint4*)(h_hi + (size_t)(from + r) * d))[i];
+        ((uint4*)(h_lo + (size_t)r * d))[i] = ((const uint4*)(h_lo + (size_t)(from + r) * d))[i];
+    }
+}
+
 // One projection of the forward.  Returns the per-tile segment counts its consumer must use.
 anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int rows, const int** seg_count_out) {
     Workspace& ws = kv->ws;
@@ -799,7 +811,14 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
         *seg_count_out = m->d_ones;
         return gemm_plain_enqueue(plan, W, a_hi, a_lo, rows, ws.part, ws.n_max_out, m->stream, &m->prof);
     }
-    ANPD_TRY(gemm_tc_enqueue(plan, W, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)ws.r_max * ws.n_max_out,
+    if (mode == 1) {                                   // a prompt pass: complete sums, one per output
+        const int n_tiles = ((plan.m_tiles + 1) / 2) * ((rows + 255) / 256);
+        const int ksplit = gemm_pf_ksplit(n_tiles, plan.k_blocks, m->num_sms);
+        *seg_count_out = m->d_const_segs[ksplit];
+        return gemm_pf_enqueue(plan, W, maps[0], maps[1], rows, ws.part, ws.n_max_out, (size_t)ws.r_max * ws.n_max_out, ksplit, m->num_sms,
+                               ws.gemm_err, m->stream, &m->prof);
+    }
+    ANPD_TRY(gemm_tc_enqueue(plan, W, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)kv->batch * ANPD_ROWS * ws.n_max_out,
                              ws.n_max_out, ws.gemm_err, m->stream, &m->prof));
     *seg_count_out = plan.d_seg_count;
     return ANPD_OK;
@@ -817,8 +836,10 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     if (first_call_on_device(attr_set)) {
         CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
+    if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && c.n_q_heads == c.n_kv_heads)
+        return attn_prompt_enqueue(m, kv, layer, rows);          // a prompt pass: pages are folded in the kernel, nothing to merge
     if (HD == 128 && kv->attn_tc) {
-        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos));
+        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos, rows != kv->batch * ANPD_ROWS));
     } else {
         dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
         LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
@@ -921,7 +942,7 @@ static anpd_status forward_rr_enqueue(anpd_model* m, anpd_kv* kv, int max_pos, b
     return ANPD_OK;
 }
 
-anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits) {
+anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits, int head_row) {
     if (m->rr_ready && kv->batch == 1 && rows == ANPD_ROWS && head && !m->plain_gemm) return forward_rr_enqueue(m, kv, max_pos, want_logits);
     if (kv->step_ready && rows == kv->batch * ANPD_ROWS && head && !m->prof.on) return step_kernel_enqueue(m, kv, max_pos, want_logits);
     const anpd_model_config& c = m->cfg;
@@ -932,7 +953,8 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     cudaStream_t st = m->stream;
     Profiler* pf = &m->prof;
     const int d = c.d_model, F = c.d_ffn, hd = c.head_dim, V = c.vocab;
-    const size_t sstride = (size_t)ws.r_max * ws.n_max_out;
+    // between the partial sums of an output: the segments of a decode step, the K parts of a prompt pass
+    const size_t sstride = (rows == kv->batch * ANPD_ROWS) ? (size_t)kv->batch * ANPD_ROWS * ws.n_max_out : (size_t)ws.r_max * ws.n_max_out;
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * hd;
     const int* segs = nullptr;
 
@@ -968,9 +990,18 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
                                                        ws.h_hi, ws.h_lo)));
     }
     if (!head) { CUDA_TRY(cudaGetLastError()); return ANPD_OK; }
-    ANPD_TRY(gemm_enqueue(m, kv, GK_LM, 0, rows, &segs));
+    int head_rows = rows;
+    if (rows != kv->batch * ANPD_ROWS) {
+        // A prompt pass needs the LM head for its last token only: the group of 8 rows that holds it moves to rows 0-7 and
+        // goes through the decode projection (the other rows of that launch are whatever the buffer holds; rows are independent).
+        head_rows = kv->batch * ANPD_ROWS;
+        LAUNCH(pf, st, KC_OTHER, 0,
+               (launch_k(move_rows_kernel, ANPD_ROWS, 256, 0, st, ws.h_hi, ws.h_lo, (head_row / ANPD_ROWS) * ANPD_ROWS, d)));
+    }
+    ANPD_TRY(gemm_enqueue(m, kv, GK_LM, 0, head_rows, &segs));
+    rows = head_rows;
     LAUNCH(pf, st, KC_OTHER, 0,
-           (launch_k(argmax_partial_kernel, dim3(ws.amax_blocks, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, V,
+           (launch_k(argmax_partial_kernel, dim3(ws.amax_blocks, rows), 256, 0, st, ws.part, segs, (size_t)kv->batch * ANPD_ROWS * ws.n_max_out, ws.n_max_out, V,
                                                                              want_logits ? ws.logits : nullptr, ws.amax_val,
                                                                              ws.amax_idx, ws.amax_blocks)));
     CUDA_TRY(cudaGetLastError());

@@ -222,7 +222,7 @@ anpd_status rr_enqueue(int epi, const RRPlan& p, const unsigned char* w, const u
 // model, KV cache and workspace
 // ---------------------------------------------------------------------------------------------
 constexpr int KV_PAGE = 128;          // positions per KV page (= key chunk of one attention block)
-constexpr int PREFILL_ROWS = 128;     // rows per prefill pass (the MMA takes hi and lo rows side by side: N = 256, its maximum)
+constexpr int PREFILL_ROWS_MAX = 2048; // most rows of one prompt pass (sizes the workspace); a longer prompt takes several passes
 
 // How one [N][K] weight matrix is cut across the persistent GEMM CTAs (depends on the shape and the
 // SM count only): tile t is started by CTA first_cta[t] and covered by seg_count[t] consecutive CTAs,
@@ -260,6 +260,7 @@ struct anpd_model {
     GemmPlan plan[GK_COUNT];
     int* d_plan_tables;               // device copies of the plans' tables
     int* d_ones;                      // [tiles] all 1: segment counts of the plain GEMM
+    int* d_const_segs[4];             // [tiles] all k (k = 1..3): segment counts of a prompt-pass GEMM cut into k parts along K
     int max_segs;
     bool plain_gemm;                  // debugging aid: route GEMMs through the plain kernel
     // second copy of the projections in row-range storage, used by single-sequence steps (proj_rr.cu)
@@ -276,6 +277,7 @@ struct anpd_model {
 
 struct Workspace {
     int r_max;                        // rows any forward may use
+    int prefill_rows;                 // rows of one prompt pass (a multiple of 256)
     int n_max_out;                    // widest GEMM output (max of nqkv, 2F, d, V)
     int splits_max;
     int* row_tok; int* row_pos; int* row_seq; int* row_ok;    // [r_max]
@@ -297,7 +299,7 @@ struct Workspace {
     int amax_nblk;                    // argmax candidates per row left by the last forward (depends on the path it took)
     float* amax_val_use; int* amax_idx_use;   // ... and the arrays that hold them
     int* gemm_err;                    // device flag set by a GEMM kernel that gave up waiting
-    // TMA views of the activation buffers: [0] decode (batch*8 rows), [1] prefill (PREFILL_ROWS rows)
+    // TMA views of the activation buffers: [0] decode (batch*8 rows), [1] prompt passes (prefill_rows rows, boxes of 128 rows)
     CUtensorMap map_h[2][2], map_ao[2][2], map_act[2][2];     // [mode][hi/lo]
     int nb[2];                        // MMA N per mode (rows padded to a multiple of 16)
 };
@@ -383,7 +385,8 @@ struct anpd_kv {
 // hold consecutive positions).  The row plan (ws.row_*) must have been written on the stream.
 // max_pos: an upper bound of the largest position any row holds (sizes the attention grid).
 // head: also run the LM head and the per-block argmax (false for all but the last prefill pass).
-anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits);
+// head_row: in a prompt pass, the row whose next token is wanted (the LM head runs for its group of 8 rows only).
+anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits, int head_row = 0);
 
 // step_kernel.cu: the whole forward of a decode step as ONE persistent kernel (one CTA per SM).  True if this model / cache
 // pair can take that path (head dimension 128, one query head per kv head, dimensions that are multiples of 128).
@@ -401,7 +404,10 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
 anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len);
 
 // attn_tc.cu: per-page attention partials for head dimension 128 (same outputs as the mma.sync kernel in forward.cu)
-anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos);
+// prompt_pass: the rows are consecutive positions of one sequence (a multiple of 8; the row plan covers the padding up to 32 rows more)
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool prompt_pass);
+// attention of a prompt pass (one query head per kv head), written straight to the O projection's input
+anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows);
 
 // gemm_tc.cu
 anpd_status make_tmap_bf16(CUtensorMap* out, const void* base, int rows, int K, int box_rows, bool streamed);
@@ -427,6 +433,11 @@ anpd_status gemm_retile_enqueue(const GemmPlan& p, const void* src, bool src_is_
 anpd_status gemm_tc_enqueue(const GemmPlan& plan, const __nv_bfloat16* w_blocks, const CUtensorMap& map_hi, const CUtensorMap& map_lo,
                             int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,
                             Profiler* prof);
+// gemm_pf.cu: the projection of a prompt pass (many rows, bound by the tensor cores): out[row][n], complete sums
+// out[part][row][n]: `ksplit` partial sums per output, seg_stride elements apart (gemm_pf_ksplit picks the cut)
+int gemm_pf_ksplit(int tiles, int k_blocks, int num_sms);
+anpd_status gemm_pf_enqueue(const GemmPlan& plan, const __nv_bfloat16* w_blocks, const CUtensorMap& map_hi, const CUtensorMap& map_lo, int rows,
+                            float* out, int ld, size_t seg_stride, int ksplit, int num_sms, int* err, cudaStream_t st, Profiler* prof);
 // forward.cu: the plain (one warp per output feature) GEMM, kept as a cross-check
 anpd_status gemm_plain_enqueue(const GemmPlan& p, const __nv_bfloat16* W, const __nv_bfloat16* a_hi, const __nv_bfloat16* a_lo, int rows,
                                float* part, int ld_part, cudaStream_t st, Profiler* prof);
