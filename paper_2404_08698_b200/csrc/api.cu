@@ -365,6 +365,16 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     kv->staged = false;
     kv->warm = false;
     kv->loop_ok = std::getenv("ANPD_HOST_LOOP") == nullptr;
+    kv->side_stream = nullptr; kv->ev_fork = nullptr; kv->ev_join = nullptr;
+    if (!m->prof.on && cudaStreamCreateWithFlags(&kv->side_stream, cudaStreamNonBlocking) == cudaSuccess) {
+        if (cudaEventCreateWithFlags(&kv->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&kv->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            if (kv->ev_fork) cudaEventDestroy(kv->ev_fork);
+            cudaStreamDestroy(kv->side_stream);
+            kv->side_stream = nullptr; kv->ev_fork = nullptr; kv->ev_join = nullptr;
+        }
+    } else cudaGetLastError();
     kv->loop_launches_per_step = 0;
     // the legacy default stream cannot be captured: steps on it are launched one kernel at a time
     kv->use_graphs = std::getenv("ANPD_NO_GRAPH") == nullptr && m->stream != nullptr && m->stream != cudaStreamLegacy;
@@ -491,6 +501,7 @@ anpd_status anpd_kv_destroy(anpd_kv* kv) {
     step_kernel_trace_dump(kv);
     for (auto& g : kv->graphs) cudaGraphExecDestroy(g.second.exec);
     for (auto& g : kv->loop_graphs) cudaGraphExecDestroy(g.second.exec);
+    if (kv->side_stream) { cudaStreamSynchronize(kv->side_stream); cudaEventDestroy(kv->ev_fork); cudaEventDestroy(kv->ev_join); cudaStreamDestroy(kv->side_stream); }
     cudaFreeHost(kv->h_seq);
     cudaFree(kv->step_slab);
     cudaFree(kv->slab);
@@ -828,10 +839,19 @@ static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* 
                                      cudaMemcpyDefault, st));
             kv->h_small[2 * b] = prompt_len; kv->h_small[2 * b + 1] = (K > 0) ? prompt_len : 0;
             CUDA_TRY(cudaMemcpyAsync(c->h.state, kv->h_small + 2 * b, 2 * sizeof(int), cudaMemcpyHostToDevice, st));
-            if (K > 0) ANPD_TRY(ngram_enqueue_bulk(c, 0, prompt_len, &m->prof));
+        }
+        // the tables are not needed before the first draft: their kernels run beside the prompt passes, on the side stream
+        if (K > 0 && kv->side_stream) {
+            CUDA_TRY(cudaEventRecord(kv->ev_fork, st));
+            CUDA_TRY(cudaStreamWaitEvent(kv->side_stream, kv->ev_fork, 0));
+            for (int b = 0; b < B; ++b) ANPD_TRY(ngram_enqueue_bulk(ctxs[b], 0, prompt_len, &m->prof, kv->side_stream));
+            CUDA_TRY(cudaEventRecord(kv->ev_join, kv->side_stream));
+        } else if (K > 0) {
+            for (int b = 0; b < B; ++b) ANPD_TRY(ngram_enqueue_bulk(ctxs[b], 0, prompt_len, &m->prof));
         }
         // LLM(prompt): the first token lands in the context as its first uncounted token
         for (int b = 0; b < B; ++b) ANPD_TRY(prefill_enqueue(m, kv, b, prompts + (size_t)b * prompt_len, prompt_len, kv->d_ctxs));
+        if (K > 0 && kv->side_stream) CUDA_TRY(cudaStreamWaitEvent(st, kv->ev_join, 0));
         CUDA_TRY(cudaEventRecord(e1, st));
         ANPD_TRY(read_seqs(kv));
         for (int b = 0; b < B; ++b) ANPD_TRY(seq_error_status(kv->h_seq[b]));

@@ -238,6 +238,85 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
     }
 }
 
+// The same for a prompt pass (rows are consecutive positions of one sequence, a multiple of 8, the first a multiple of 64):
+// a block takes 64 rows of one head through shared memory, so that the transposed V page receives whole 16-byte runs of
+// positions instead of single elements.  Per element the arithmetic is that of qkv_rope_append_kernel, in the same order.
+constexpr int ROPE_TILE_ROWS = 64;
+template <int HD>
+__global__ void __launch_bounds__(256) qkv_rope_append_tile_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride,
+                                                                   int ld_part, int rows, const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                                                                   const int* __restrict__ row_ok, const float* __restrict__ rope_cos,
+                                                                   const float* __restrict__ rope_sin, const int* __restrict__ page_table,
+                                                                   int pages_per_seq, int Hq, int Hkv, float q_scale, bf16* __restrict__ q_hi,
+                                                                   bf16* __restrict__ q_lo, bf16* __restrict__ kpool_l, bf16* __restrict__ vpool_l) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float tile[ROPE_TILE_ROWS][HD + 1];
+    constexpr int half = HD / 2;
+    const int r0 = blockIdx.x * ROPE_TILE_ROWS, head = blockIdx.y;
+    const int nr = min(ROPE_TILE_ROWS, rows - r0);
+    const int ns = seg_count[(head * HD) >> 7];          // a head never straddles a 128-column tile
+    // 16-byte loads, eight of them in flight per thread
+    constexpr int Q4 = HD / 4;
+#pragma unroll 8
+    for (int idx = threadIdx.x; idx < nr * Q4; idx += 256) {
+        const int r = idx / Q4, dim = (idx % Q4) * 4;
+        const float* pr = part + (size_t)(r0 + r) * ld_part + (size_t)head * HD + dim;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < ns; ++s) { const float4 v = *(const float4*)(pr + s * split_stride); a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+        tile[r][dim] = a.x; tile[r][dim + 1] = a.y; tile[r][dim + 2] = a.z; tile[r][dim + 3] = a.w;
+    }
+    __syncthreads();
+    if (head < Hq + Hkv) {
+        for (int idx = threadIdx.x; idx < nr * half; idx += 256) {
+            const int r = idx / half, i = idx % half;
+            const int pos = row_pos[r0 + r];
+            const float a = tile[r][i], b = tile[r][i + half];
+            const float c = rope_cos[(size_t)pos * half + i], sn = rope_sin[(size_t)pos * half + i];
+            tile[r][i] = a * c - b * sn;
+            tile[r][i + half] = b * c + a * sn;
+        }
+        __syncthreads();
+    }
+    if (head < Hq) {
+        for (int idx = threadIdx.x; idx < nr * Q4; idx += 256) {
+            const int r = idx / Q4, dim = (idx % Q4) * 4;
+            const size_t o = (size_t)(r0 + r) * Hq * HD + (size_t)head * HD + dim;
+            store_split4(make_float4(tile[r][dim] * q_scale, tile[r][dim + 1] * q_scale, tile[r][dim + 2] * q_scale, tile[r][dim + 3] * q_scale),
+                         q_hi + o, q_lo + o);
+        }
+        return;
+    }
+    const bool is_k = head < Hq + Hkv;
+    const int kvh = is_k ? head - Hq : head - Hq - Hkv;
+    const int pos0 = row_pos[r0];                        // the tile's rows hold positions pos0, pos0 + 1, ... inside one page
+    const int page = page_table[row_seq[r0] * pages_per_seq + pos0 / KV_PAGE];
+    bf16* pg = (is_k ? kpool_l : vpool_l) + ((size_t)page * Hkv + kvh) * KV_PAGE * HD;
+    if (is_k) {                                          // K page: [position][dim]
+        for (int idx = threadIdx.x; idx < nr * Q4; idx += 256) {
+            const int r = idx / Q4, dim = (idx % Q4) * 4;
+            if (!row_ok[r0 + r]) continue;
+            bf16 v[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[e] = __float2bfloat16_rn(tile[r][dim + e]);
+            *(uint2*)(pg + (size_t)((pos0 + r) % KV_PAGE) * HD + dim) = *(const uint2*)v;
+        }
+    } else {                                             // V page, transposed: [dim][position]; 8 positions = 16 bytes
+        for (int idx = threadIdx.x; idx < (ROPE_TILE_ROWS / 8) * HD; idx += 256) {
+            const int dim = idx % HD, r8 = (idx / HD) * 8;
+            if (r8 >= nr) continue;
+            bf16 v[8];
+            bool all = true;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { v[e] = __float2bfloat16_rn(tile[r8 + e][dim]); all = all && row_ok[r0 + r8 + e] != 0; }
+            bf16* dst = pg + (size_t)dim * KV_PAGE + (pos0 % KV_PAGE) + r8;
+            if (all) *(uint4*)dst = *(const uint4*)v;
+            else
+                for (int e = 0; e < 8; ++e) if (row_ok[r0 + r8 + e]) dst[e] = v[e];
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // attention: per (key page, kv head, group of 8 rows) partial softmax, then a combine in page order
 //
@@ -965,6 +1044,18 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& w = m->layers[l];
         ANPD_TRY(gemm_enqueue(m, kv, GK_QKV, l, rows, &segs));
+        if (rows != kv->batch * ANPD_ROWS) {            // a prompt pass
+            const dim3 grid((rows + ROPE_TILE_ROWS - 1) / ROPE_TILE_ROWS, c.n_q_heads + 2 * c.n_kv_heads);
+            const float qs = 1.4426950408889634f / sqrtf((float)hd);
+            if (hd == 128) LAUNCH(pf, st, KC_OTHER, 0,
+                   (launch_k(qkv_rope_append_tile_kernel<128>, grid, 256, 0, st, ws.part, segs, sstride, ws.n_max_out, rows, ws.row_pos, ws.row_seq, ws.row_ok,
+                             kv->rope_cos, kv->rope_sin, kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, qs, ws.q_hi, ws.q_lo,
+                             kv->kpool + l * layer_elems, kv->vpool + l * layer_elems)));
+            else LAUNCH(pf, st, KC_OTHER, 0,
+                   (launch_k(qkv_rope_append_tile_kernel<64>, grid, 256, 0, st, ws.part, segs, sstride, ws.n_max_out, rows, ws.row_pos, ws.row_seq, ws.row_ok,
+                             kv->rope_cos, kv->rope_sin, kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, qs, ws.q_hi, ws.q_lo,
+                             kv->kpool + l * layer_elems, kv->vpool + l * layer_elems)));
+        } else
         LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(qkv_rope_append_kernel, dim3(rows, (c.n_q_heads + 2 * c.n_kv_heads + rope_hpb - 1) / rope_hpb), rope_hpb * (hd / 2), 0, st, 
                    ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,

@@ -165,7 +165,8 @@ struct anpd_ngram {
     size_t slab_bytes;
 };
 
-anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof);
+// on: the stream to launch on (null: the context's own)
+anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof, cudaStream_t on = nullptr);
 // One fused launch for `batch` sequences: folds tokens [state[1], state[0]) of each, then drafts
 // K tokens into seq[b] (draft, draft_len, last_tok).
 anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batch, int K,
@@ -370,6 +371,9 @@ struct anpd_kv {
     std::map<uint64_t, StepGraph> loop_graphs;
     bool loop_ok;                     // false once building such a graph has failed, or when ANPD_HOST_LOOP is set
     int* loop_steps_left;             // device: steps the running loop may still take
+    // Initialize (the prompt's n-gram statistics) runs on a stream of its own under the prompt passes
+    cudaStream_t side_stream;
+    cudaEvent_t ev_fork, ev_join;
     int loop_launches_per_step;
     // persistent step kernel: its arguments, the buffers only it uses, and whether decode steps take it
     StepParams step;

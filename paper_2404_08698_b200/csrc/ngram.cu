@@ -186,14 +186,15 @@ int next_pow2(int v) { int p = 64; while (p < v) p <<= 1; return p; }
 
 }  // namespace
 
-anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof) {
+anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof, cudaStream_t on) {
     if (to <= from) return ANPD_OK;
+    cudaStream_t st = on ? on : ctx->stream;
     const int levels = ctx->h.n_max - ctx->h.n_min + 1;
     const int items = (to - from) * levels;
     const int threads = 256, wpb = threads / 32;
     const int blocks = std::min((items + wpb - 1) / wpb, 148 * 8);
-    LAUNCH(prof, ctx->stream, KC_NGRAM, 0, (ngram_bulk_kernel<1><<<blocks, threads, 0, ctx->stream>>>(ctx->h, from, to)));
-    LAUNCH(prof, ctx->stream, KC_NGRAM, 0, (ngram_bulk_kernel<2><<<blocks, threads, 0, ctx->stream>>>(ctx->h, from, to)));
+    LAUNCH(prof, st, KC_NGRAM, 0, (ngram_bulk_kernel<1><<<blocks, threads, 0, st>>>(ctx->h, from, to)));
+    LAUNCH(prof, st, KC_NGRAM, 0, (ngram_bulk_kernel<2><<<blocks, threads, 0, st>>>(ctx->h, from, to)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
