@@ -38,6 +38,29 @@ HBM_NOMINAL_GBS = 8000.0          # the roofline the target is stated against
 HBM_FALLBACK_GBS = 6650.0         # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
 
 
+def measured_tensor_peak() -> tuple[float, str]:
+    """Sustained dense bf16 TFLOP/s of this machine's B200s (a long cuBLAS loop under the power cap), else the recipe's fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1400.0, "fallback"
+
+
+def prefill_summary(wl, ms_prefill: float) -> dict:
+    """The prompt passes against the tensor-core roofline: every projection of every layer over all prompt rows (the LM head runs
+    for the last token only and is left out, as is attention).  The activations enter as two bf16 terms (hi + lo), so the MMAs
+    do twice the useful FLOPs; both rates are given."""
+    s = wl.shape
+    proj = s.streamed_params - s.vocab * s.d_model
+    useful = 2.0 * wl.prompt_len * proj * wl.batch
+    peak, kind = measured_tensor_peak()
+    t = ms_prefill * 1e-3
+    return {"ms": ms_prefill, "rows": wl.prompt_len * wl.batch, "useful_tflops": useful / t / 1e12, "mma_tflops_hi_plus_lo": 2.0 * useful / t / 1e12,
+            "peak_tflops": peak, "peak_kind": f"of {kind} (sustained)", "frac_mma_of_peak": 2.0 * useful / t / 1e12 / peak}
+
+
 def measured_hbm_peak() -> tuple[float, str]:
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -685,6 +708,7 @@ def main() -> None:
         "anpd_equals_greedy": lossless,
         "verify_step": {"kv_len": P, "rows": A.ROWS, "ms": ms_verify, "bytes": step_bytes, "gbs": verify_gbs,
                         "frac_of_8TBs": verify_gbs / HBM_NOMINAL_GBS, f"frac_of_{peak_kind}_copy": verify_gbs / peak},
+        "prefill": prefill_summary(wl, st_anpd["ms_prefill"]),
         "setup_s": t_setup,
     }
     # ---- n-gram kernels alone (update + draft of one step), from an event-bracketed (eager) short run ---------------
