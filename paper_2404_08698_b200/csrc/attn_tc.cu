@@ -70,10 +70,7 @@ __device__ __forceinline__ void slot_bar(int slot) { asm volatile("bar.sync %0, 
 
 struct AttnItem { int c, kvh, r0, pos_lo, seq; };
 
-// PF (prompt passes of a model with one query head per kv head): an item's 8 x G query vectors are 8 x G consecutive rows of ONE
-// head (consecutive positions of the prompt) instead of 8 rows of G heads, so a page is fetched once for 8 x G rows; AttnItem::kvh
-// then holds the head.
-template <int G, int S, bool PF>
+template <int G, int S>
 __global__ void __launch_bounds__(AttnCfg<G, S>::THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const bf16* __restrict__ q_hi,
                const bf16* __restrict__ q_lo, const int* __restrict__ page_table, int pages_per_seq, const int* __restrict__ row_pos,
@@ -121,12 +118,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     const int stride = gridDim.x * SLOTS;
     auto decode = [&](int it, AttnItem& out) {
         const int rest = it / chunks;
-        out.c = it % chunks; out.kvh = rest % Hkv; out.r0 = (rest / Hkv) * (PF ? Q : ANPD_ROWS);
+        out.c = it % chunks; out.kvh = rest % Hkv; out.r0 = (rest / Hkv) * ANPD_ROWS;
     };
     auto next_item = [&](int it, AttnItem& out) -> int {
         for (; it < n_items; it += stride) {
             decode(it, out);
-            const int hi = row_pos[out.r0 + (PF ? Q : ANPD_ROWS) - 1];   // three independent loads
+            const int hi = row_pos[out.r0 + ANPD_ROWS - 1];          // three independent loads
             out.pos_lo = row_pos[out.r0];
             out.seq = row_seq[out.r0];
             if (out.c * KV_PAGE <= hi) return it;
@@ -151,8 +148,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             if (idx < N * 16) {
                 const int n = idx >> 4, c16 = idx & 15;
                 const int qn = n % Q, g = qn >> 3, r = qn & 7;
-                const bf16* src = (n < Q ? q_hi : q_lo) + (PF ? (size_t)(a.r0 + qn) * Hq * HD + (size_t)a.kvh * HD
-                                                              : (size_t)(a.r0 + r) * Hq * HD + (size_t)(a.kvh * G + g) * HD) + c16 * 8;
+                const bf16* src = (n < Q ? q_hi : q_lo) + (size_t)(a.r0 + r) * Hq * HD + (size_t)(a.kvh * G + g) * HD + c16 * 8;
                 regs[u] = *(const uint4*)src;
             }
         }
@@ -219,7 +215,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         const int key = cur.c * KV_PAGE + t;
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
-            if (key > cur.pos_lo + (PF ? q : (q & 7))) s[q] = -CUDART_INF_F;
+            if (key > cur.pos_lo + (q & 7)) s[q] = -CUDART_INF_F;
             float mx = s[q];
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if (lane == 0) red_max[slot][warp][q] = mx;
@@ -257,7 +253,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             }
         }
         if (t < Q) {
-            const size_t out = (PF ? (size_t)(cur.r0 + t) * Hq + cur.kvh : (size_t)(cur.r0 + (t & 7)) * Hq + (cur.kvh * G + (t >> 3))) * pages_per_seq + cur.c;
+            const size_t out = ((size_t)(cur.r0 + (t & 7)) * Hq + (cur.kvh * G + (t >> 3))) * pages_per_seq + cur.c;
             float mt = m[0];
 #pragma unroll
             for (int q = 1; q < Q; ++q) mt = (q == t) ? m[q] : mt;
@@ -273,7 +269,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
             for (int c0 = 0; c0 < N; c0 += 16) tc_ld16(lane_base + (uint32_t)c0, v + c0);
 #pragma unroll
             for (int q = 0; q < Q; ++q) {
-                const size_t out = (PF ? (size_t)(cur.r0 + q) * Hq + cur.kvh : (size_t)(cur.r0 + (q & 7)) * Hq + (cur.kvh * G + (q >> 3))) * pages_per_seq + cur.c;
+                const size_t out = ((size_t)(cur.r0 + (q & 7)) * Hq + (cur.kvh * G + (q >> 3))) * pages_per_seq + cur.c;
                 po[out * HD + t] = v[q] + v[Q + q];
             }
         }
@@ -500,21 +496,21 @@ attn_prompt_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
 }
 
-template <int G, int S, bool PF = false>
+template <int G, int S>
 anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int chunks) {
     typedef AttnCfg<G, S> Cfg;
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
     static bool attr_set[64] = {false};
     if (first_call_on_device(attr_set)) {
-        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G, S, PF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        CUDA_TRY(cudaFuncSetAttribute(attn_tc_kernel<G, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
     }
     const int layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
-    const int n_items = PF ? chunks * c.n_q_heads * ((rows + Cfg::Q - 1) / Cfg::Q) : chunks * c.n_kv_heads * (rows / ANPD_ROWS);
+    const int n_items = chunks * c.n_kv_heads * (rows / ANPD_ROWS);
     const int grid = std::min(m->num_sms, n_items);
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_tc_kernel<G, S, PF>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
-                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, PF ? c.n_q_heads : c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
+           (launch_k(attn_tc_kernel<G, S>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
+                     kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
                      ws.attn_l, ws.attn_o, ws.gemm_err)));
     return ANPD_OK;
 }
@@ -540,12 +536,8 @@ anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows)
     return ANPD_OK;
 }
 
-anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool prompt_pass) {
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos) {
     const int chunks = max_pos / KV_PAGE + 1;
-    if (prompt_pass && m->cfg.n_q_heads == m->cfg.n_kv_heads) {
-        // rows are consecutive positions of one sequence: 16 of them share every page fetch (32 or 64 rows per item measured slower)
-        return launch_attn_tc<2, 4, true>(m, kv, layer, rows, chunks);
-    }
     const int n_items = chunks * m->cfg.n_kv_heads * (rows / ANPD_ROWS);
     switch (m->cfg.n_q_heads / m->cfg.n_kv_heads) {
         // one query head per kv head fits five slots; while every item finds a slot with four, four are faster

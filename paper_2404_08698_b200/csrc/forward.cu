@@ -918,7 +918,7 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && c.n_q_heads == c.n_kv_heads)
         return attn_prompt_enqueue(m, kv, layer, rows);          // a prompt pass: pages are folded in the kernel, nothing to merge
     if (HD == 128 && kv->attn_tc) {
-        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos, rows != kv->batch * ANPD_ROWS));
+        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos));
     } else {
         dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
         LAUNCH(&m->prof, m->stream, KC_ATTN, 0,

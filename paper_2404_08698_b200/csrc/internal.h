@@ -408,8 +408,7 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
 anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len);
 
 // attn_tc.cu: per-page attention partials for head dimension 128 (same outputs as the mma.sync kernel in forward.cu)
-// prompt_pass: the rows are consecutive positions of one sequence (a multiple of 8; the row plan covers the padding up to 32 rows more)
-anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool prompt_pass);
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos);
 // attention of a prompt pass (one query head per kv head), written straight to the O projection's input
 anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows);
 

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import as_bf16_values, gpu_model, require_gpu, top2_margin
+from helpers import as_bf16_values, gpu_model, new_stream, require_gpu, top2_margin
 from oracle.anpd import accept_length, argmax_lowest
 from oracle.decoder import Decoder
 from workloads import WORKLOADS, ModelShape, make_prompts, make_weights, markov_prompt
@@ -310,3 +310,32 @@ def test_row_range_projections_logits_parity(A, monkeypatch, shape, plen):
         assert A.anpd_kv_len(r.kv) == plen + acc + 1
     finally:
         r.close()
+
+
+@pytest.mark.parametrize("shape,plen", [
+    (ModelShape(2, 256, 2, 2, 128, 688, 4096), 2050),      # head dimension 128, one query head per kv head: the prompt kernels
+    (ModelShape(2, 256, 4, 2, 64, 688, 4096), 2101),       # head dimension 64, grouped heads: page partials and their merge
+], ids=["hd128", "hd64"])
+def test_prompt_longer_than_one_pass(A, shape, plen):
+    """A prompt of more than 2048 tokens takes two prompt passes; the second is short (2 and 53 tokens: 8 and 56 rows) and
+    attends to the pages the first one wrote.  First token and the logits of a verify step after it against the oracle."""
+    w = make_weights(shape, 5, False, std=0.05)
+    prompt = markov_prompt(plen, shape.vocab, 2, 77).tolist()
+    draft = [int(t) for t in markov_prompt(7, shape.vocab, 2, 78)]
+    m = gpu_model(A, shape, w, new_stream())
+    kv = A.anpd_kv_create(m, plen + 64)
+    try:
+        first = A.anpd_prefill(m, kv, prompt)
+        got = A.anpd_verify_logits(m, kv, first, draft, shape.vocab)
+    finally:
+        A.anpd_kv_destroy(kv)
+        A.anpd_model_destroy(m)
+    dec = Decoder(shape, as_bf16_values(w), torch.float64, kv_dtype=torch.bfloat16)
+    cache = dec.new_cache()
+    lp = dec.forward(prompt, cache)
+    if top2_margin(lp[-1]) > 5e-2:
+        assert first == argmax_lowest(lp[-1])
+    want = dec.forward([first] + draft, cache)
+    err = float((torch.from_numpy(got).double() - want).abs().max())
+    print(f"{plen} tokens, hd {shape.head_dim}: max-abs {err:.2e}")
+    assert err <= 5e-3, err
