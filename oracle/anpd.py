@@ -92,6 +92,62 @@ def speedup_bound(alpha: float, K: int) -> float:
     return alpha * K + 1.0
 
 
+def two_candidate_lengths(K: int) -> tuple[int, int]:
+    """Draft lengths of the two candidates of a step when a step has room for 7 draft rows: the first
+    candidate keeps up to 4 tokens, the alternative up to 3 (both at most K)."""
+    return min(K, 4), min(K, 3)
+
+
+def anpd_generate_two_candidates(model, prompt, max_new: int, K: int, n_max: int = 5, n_min: int = 2,
+                                 policy: int = POLICY_MAX_COUNT):
+    """Algorithm 1 with two candidates per step (the conclusion's future-work item: several candidates verified
+    at once).  Each step drafts the usual candidate A and an alternative B (MLN.draft_alternative), verifies
+    both against the same cache state - written here as two forwards from the same state; one forward with a tree
+    mask computes the same rows - and keeps the one with the longer accepted prefix (A on a tie).  The output is
+    still the model's greedy output.  Returns (tokens[:max_new], Stats, mln); Stats.drafted counts the tokens of
+    both candidates, Stats.drafts holds (A, B) per step and Stats.alt_wins the steps B won."""
+    mln = MLN(n_min, n_max, policy)
+    mln.initialize(prompt)
+    st = Stats()
+    st.alt_wins = 0
+    ka, kb = two_candidate_lengths(K)
+    cache = model.new_cache()
+    logits = model.forward(list(prompt), cache)
+    confirmed = argmax_lowest(logits[-1])
+    out: list[int] = []
+    while len(out) < max_new:
+        out.append(confirmed)
+        mln.update(confirmed)
+        da = mln.draft(ka)
+        db = mln.draft_alternative(da[0] if da else None, kb)
+        P = cache.length
+        a_a, nxt_a, _, _ = verify(model, cache, confirmed, da)
+        a_b, nxt_b = 0, None
+        if db:
+            cache.truncate(P)
+            a_b, nxt_b, _, _ = verify(model, cache, confirmed, db)
+        if a_b > a_a:
+            chosen, a, nxt = db, a_b, nxt_b
+            st.alt_wins += 1
+        else:
+            chosen, a, nxt = da, a_a, nxt_a
+            if db:                                       # the cache holds B's rows: put A's accepted rows back
+                cache.truncate(P)
+                verify(model, cache, confirmed, da[:a_a])
+        for tok in chosen[:a]:
+            out.append(tok)
+            mln.update(tok)
+        st.steps += 1
+        st.drafted += len(da) + len(db)
+        st.accepted += a
+        st.hist_accepted[a] += 1
+        st.drafts.append((list(da), list(db)))
+        st.accepted_lens.append(a)
+        confirmed = nxt
+    st.generated = len(out)
+    return out[:max_new], st, mln
+
+
 def anpd_generate(model, prompt, max_new: int, K: int, n_max: int = 5, n_min: int = 2,
                   policy: int = POLICY_MAX_COUNT, mln: MLN | None = None):
     """Algorithm 1.  Returns (tokens[:max_new], Stats, mln)."""

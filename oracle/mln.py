@@ -90,6 +90,30 @@ class MLN:
             ctx.append(s)
         return out
 
+    def draft_alternative(self, first: int | None, K: int) -> list[int]:
+        """A second candidate for the same step (the paper's conclusion names verifying several candidates at
+        once as future work; this is the reading taken here).  Its first token is the answer of the highest
+        level whose answer DIFFERS from `first` (the first token of `draft`): where the longest matching context
+        and a shorter one disagree about the next token, the shorter one's answer is the alternative.  The
+        candidate then continues like `draft`, by chained back-off queries on its own temporary context, up to
+        K tokens in all.  Empty if K is 0, if `first` is None (nothing was drafted) or if no level disagrees."""
+        if K <= 0 or first is None:
+            return []
+        ctx = list(self.tokens[-(self.n_max - 1):]) if self.n_max > 1 else []
+        answers = (self.query_level(n, ctx) for n in range(self.n_max, self.n_min - 1, -1))
+        alt = next((a for a in answers if a is not None and a != int(first)), None)
+        if alt is None:
+            return []
+        out = [alt]
+        ctx.append(alt)
+        while len(out) < K:
+            s = self.query(ctx)
+            if s is None:
+                break
+            out.append(s)
+            ctx.append(s)
+        return out
+
     # -- canonical dumps, for comparing with another implementation ----------
     def dump(self, n: int) -> list[tuple[tuple, int, int, int]]:
         """Every level-n record as (context, successor, count, last_pos), sorted."""

@@ -7,7 +7,8 @@ import random
 import pytest
 import torch
 
-from oracle.anpd import (accept_length, anpd_generate, argmax_lowest, greedy, speedup_bound, verify)
+from oracle.anpd import (accept_length, anpd_generate, anpd_generate_two_candidates, argmax_lowest, greedy, speedup_bound,
+                         two_candidate_lengths, verify)
 from oracle.decoder import Decoder
 from oracle.mln import POLICY_LAST_SEEN, POLICY_MAX_COUNT
 from workloads import ModelShape, WORKLOADS, make_prompts, make_weights, periodic_prompt
@@ -173,3 +174,40 @@ def test_full_drafts_mean_tokens_per_step_is_one_plus_alpha_K():
     assert out == greedy(model, prompt, 90)
     if all(len(d) == K for d in st.drafts):
         assert abs(st.generated / st.steps - speedup_bound(st.hit_ratio, K)) < 1e-12
+
+
+@pytest.mark.parametrize("policy", [POLICY_MAX_COUNT, POLICY_LAST_SEEN])
+def test_two_candidates_are_lossless_and_never_slower_per_step(policy):
+    """Two candidates per step: the output is still the greedy output for every K and N; each step commits at least
+    what the first candidate alone would have committed from the same state (so never more steps than with the first
+    candidate's length alone), the alternative wins somewhere, and drafted counts both candidates."""
+    def fn(h):
+        return (h[-1] * 7 + (h[-2] if len(h) > 1 else 0) * 3 + (len(h) % 5 == 0)) % 6
+    model = ScriptedModel(6, fn)
+    prompt = [1, 4, 2, 2, 5, 0, 3, 1, 4, 2]
+    want = greedy(model, prompt, 80)
+    wins = 0
+    for K in range(0, 8):
+        ka, kb = two_candidate_lengths(K)
+        assert ka <= 4 and kb <= 3 and ka + kb <= 7 and ka <= K and kb <= K
+        for N in range(2, 8):
+            out, st, _ = anpd_generate_two_candidates(model, prompt, 80, K, n_max=N, policy=policy)
+            assert out == want, (K, N)
+            assert st.generated == st.steps + st.accepted and st.generated >= 80
+            assert all(len(a) <= ka and len(b) <= kb for a, b in st.drafts)
+            assert all(not b or (a and b[0] != a[0]) for a, b in st.drafts)
+            assert st.drafted == sum(len(a) + len(b) for a, b in st.drafts)
+            one, st1, _ = anpd_generate(model, prompt, 80, ka, n_max=N, policy=policy)
+            assert one == want and st.steps <= st1.steps, (K, N, st.steps, st1.steps)
+            wins += st.alt_wins
+    assert wins > 0
+
+
+def test_two_candidates_on_tiny_decoder():
+    wl = WORKLOADS["C1"]
+    w = make_weights(wl.shape, wl.weight_seed, wl.weights_bf16)
+    dec = Decoder(wl.shape, w, torch.float64)
+    prompt = make_prompts(wl)[0].tolist()
+    want = greedy(dec, prompt, 24)
+    out, st, _ = anpd_generate_two_candidates(dec, prompt, 24, 4, n_max=3)
+    assert out == want and st.generated == st.steps + st.accepted

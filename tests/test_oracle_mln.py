@@ -161,3 +161,65 @@ def test_hand_worked_example():
     b.initialize(g["tokens2"])
     assert a.draft(1) == g["first_draft_max_count"]
     assert b.draft(1) == g["first_draft_last_seen"]
+
+
+def brute_level_answer(tokens, ctx, n, policy):
+    """Answer of level n alone, by string search: best successor of the last n-1 tokens of ctx in `tokens`."""
+    if len(ctx) < n - 1:
+        return None
+    key = list(ctx[len(ctx) - (n - 1):])
+    cands = {}
+    for t in range(n - 1, len(tokens)):
+        if tokens[t - n + 1:t] == key:
+            c, _ = cands.get(tokens[t], (0, -1))
+            cands[tokens[t]] = (c + 1, t)
+    if not cands:
+        return None
+    if policy == POLICY_MAX_COUNT:
+        return max(cands, key=lambda s: cands[s])
+    return max(cands, key=lambda s: cands[s][1])
+
+
+@pytest.mark.parametrize("policy", [POLICY_MAX_COUNT, POLICY_LAST_SEEN])
+@pytest.mark.parametrize("seed", range(12))
+def test_alternative_draft_equals_bruteforce(seed, policy):
+    """The second candidate of a step: its first token is what the longest level that DISAGREES with the first
+    candidate's first token proposes (string search per level); it continues by ordinary back-off queries."""
+    rng = random.Random(500 + seed)
+    V, T, N = rng.choice([2, 3, 4]), rng.randint(4, 48), rng.randint(2, 6)
+    toks = [rng.randrange(V) for _ in range(T)]
+    m = MLN(2, N, policy)
+    m.initialize(toks)
+    first = m.draft(1)
+    assert m.draft_alternative(first[0] if first else None, 0) == []
+    assert m.draft_alternative(None, 3) == []
+    got = m.draft_alternative(first[0] if first else None, 3)
+    want = []
+    if first:
+        alt = None
+        for n in range(N, 1, -1):
+            a = brute_level_answer(toks, toks, n, policy)
+            if a is not None and a != first[0]:
+                alt = a
+                break
+        if alt is not None:
+            want, ctx = [alt], list(toks) + [alt]
+            while len(want) < 3:
+                s = brute_query(toks, ctx, 2, N, policy)
+                if s is None:
+                    break
+                want.append(s)
+                ctx.append(s)
+    assert got == want
+    assert not got or got[0] != first[0]
+    assert m.tokens == toks
+
+
+def test_alternative_draft_hand_case():
+    # after "... 7": the trigram context (5, 7) was followed by 1; the bigram context (7) by 1 once and by 2 twice
+    toks = [5, 7, 1, 9, 7, 2, 8, 7, 2, 5, 7]
+    m = MLN(2, 3)
+    m.initialize(toks)
+    assert m.draft(1) == [1]                      # longest level wins
+    assert m.draft_alternative(1, 1) == [2]       # the bigram level disagrees
+    assert m.draft_alternative(2, 1) == [1]       # had 2 been drafted, the trigram level would be the one that differs
