@@ -510,6 +510,52 @@ def ablation_sweep(args, A, wl, model, stream) -> None:
                 print(f"  {N:>3d} " + "".join(f"  {r['speedup_vs_greedy']:5.2f} ({r['hit_ratio_alpha']:4.2f})" for r in cells), file=sys.stderr)
 
 
+def two_candidate_bench(args, A, wl, model, stream) -> None:
+    """One candidate per step against two (anpd_kv_set_candidates) on an orbit workload, with the workload's own prompt
+    (random corruptions: no n-gram level is better than the longest) and with a forked prompt (workloads.orbit_fork_prompt:
+    the long contexts mislead, the shortest is right).  Every run goes through anpd_generate_dev; prints one JSON line."""
+    from workloads import orbit_continuation, orbit_fork_prompt, orbit_permutation, orbit_prompt
+    if wl.orbit_S == 0:
+        raise SystemExit("--mode candidates needs an orbit workload: e.g. --workload C3-A20")
+    pi = orbit_permutation(wl.orbit_S, wl.weight_seed)
+    max_len = wl.prompt_len + wl.max_new + 64
+    kv = A.anpd_kv_create(model, max_len)
+    ctx = A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, stream.cuda_stream)
+    out_dev = torch.zeros(wl.max_new, dtype=torch.int32, device="cuda")
+    rows, reps = [], max(args.steps, 1)
+    prompts = {"corrupted prompt": orbit_prompt(pi, wl.prompt_len, wl.corrupt, wl.prompt_seed),
+               "forked prompt": orbit_fork_prompt(pi, wl.prompt_len, wl.prompt_seed)}
+    for kind, prompt in prompts.items():
+        want = orbit_continuation(pi, prompt[-1], wl.max_new)
+        prompt_dev = torch.from_numpy(prompt).cuda()
+        for label, cands, K in (("greedy", 1, 0), (f"one candidate, K={wl.K}", 1, wl.K), ("one candidate, K=4", 1, 4),
+                                ("two candidates, 4+3", 2, max(wl.K, 4))):
+            A.anpd_kv_set_candidates(kv, cands)
+            A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            t = e0.elapsed_time(e1) / 1e3 / reps
+            rows.append({"prompt": kind, "mode": label, "tokens_per_s": wl.max_new / t, "steps": st["steps"], "drafted": st["drafted"],
+                         "accepted": st["accepted"], "alt_wins": st["alt_wins"], "ms_per_step": st["ms_decode"] / st["steps"],
+                         "equals_closed_form": bool(np.array_equal(out_dev.cpu().numpy(), want))})
+    A.anpd_kv_set_candidates(kv, 1)
+    A.anpd_ngram_destroy(ctx)
+    A.anpd_kv_destroy(kv)
+    best = max(r["tokens_per_s"] for r in rows if r["mode"].startswith("two"))
+    print(json.dumps({"metric": "tokens_per_s_two_candidates", "value": best, "unit": "tokens/s (best two-candidate row)",
+                      "higher_is_better": True, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"{wl.name}: orbit model at {wl.shape.n_layers}L d{wl.shape.d_model}, prompt {wl.prompt_len}, "
+                                             f"{wl.max_new} new tokens, N={wl.n_max}", "reps": reps}, "rows": rows}))
+    for r in rows:
+        print(f"  {r['prompt']:>17s}  {r['mode']:>22s}  {r['tokens_per_s']:8.1f} tok/s  {r['steps']:4d} steps  {r['ms_per_step']:.3f} ms/step  "
+              f"second candidate won {r['alt_wins']}", file=sys.stderr)
+
+
 def job_time_and_value(dist, seconds: float, units_per_rank: float, world: int, device) -> tuple[float, float]:
     """Replicas only: the job's time is the slowest rank's, its value the units of all ranks over that
     time.  `dist` is torch.distributed (or None for one process)."""
@@ -530,9 +576,9 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-structured", action="store_true", help="skip the orbit-model runs that follow the C3 line")
     ap.add_argument("--verify-iters", type=int, default=40)
-    ap.add_argument("--mode", default="generate", choices=["generate", "verify", "sweep"],
+    ap.add_argument("--mode", default="generate", choices=["generate", "verify", "sweep", "candidates"],
                     help="verify: the verify-step microbenchmark only (KV length, widths, forced acceptance); "
-                         "sweep: K x N x back-off x policy on an orbit workload")
+                         "sweep: K x N x back-off x policy on an orbit workload; candidates: one against two candidates per step")
     ap.add_argument("--sweep-K", type=int, nargs="+", default=[1, 2, 3, 4, 5, 6, 7])
     ap.add_argument("--sweep-N", type=int, nargs="+", default=[2, 3, 4, 5, 6, 7])
     ap.add_argument("--kv-len", type=int, nargs="+", default=[2048, 4096])
@@ -576,6 +622,10 @@ def main() -> None:
         return
     if args.mode == "sweep":
         ablation_sweep(args, A, wl, model, stream)
+        A.anpd_model_destroy(model)
+        return
+    if args.mode == "candidates":
+        two_candidate_bench(args, A, wl, model, stream)
         A.anpd_model_destroy(model)
         return
     if wl.batch > 1:

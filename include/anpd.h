@@ -97,6 +97,8 @@ typedef struct {
     int accepted;         /* draft tokens accepted; hit ratio alpha = accepted / drafted (Sec. 4.4) */
     int generated;        /* tokens committed by the loop (may exceed max_new by up to K) */
     int hist_accepted[8]; /* steps by accepted_len */
+    int alt_wins;         /* two-candidate mode: steps whose second candidate was the one kept (else 0) */
+    int reserved;
     double ms_prefill;    /* device time of the prompt forward (CUDA events) */
     double ms_decode;     /* device time of the decoding loop, first step to last */
     double bytes_per_step;/* weight + KV bytes one verify step must read, at the mean KV length */
@@ -141,6 +143,16 @@ anpd_status anpd_kv_len(anpd_kv* kv, int seq, int* len);
  * entries past `len` are simply overwritten by later steps (Section 3.1: rejected tokens
  * and everything after them are discarded). */
 anpd_status anpd_kv_truncate(anpd_kv* kv, int seq, int len);
+/* Candidates verified per step of the decoding loops (anpd_generate*): 1 (Algorithm 1 as printed) or 2.  The Conclusion
+ * names, as future work, verifying several draft candidates in parallel; with 2, a step drafts the usual candidate (cut
+ * to min(K, 4) tokens) and a second one of up to min(K, 3) tokens whose first token is the answer of the longest N-gram
+ * level that disagrees with the first candidate's first token (continued by ordinary back-off queries; empty when no
+ * level disagrees).  Both are verified by the same forward over the step's 8 rows - the second candidate's rows attend to
+ * the committed context and to themselves, not to the first candidate - and the one with the longer accepted prefix is
+ * committed (the first on a tie).  The output stays the model's greedy output.  anpd_stats.drafted then counts the tokens
+ * of both candidates and anpd_stats.alt_wins the steps the second one won.  The staged verify calls (anpd_verify*) always
+ * take one candidate.  ANPD_ERR_RANGE for any other value. */
+anpd_status anpd_kv_set_candidates(anpd_kv* kv, int candidates);
 
 /* ---- N-gram module (Sections 3.1, 3.2) ---------------------------------------------------- */
 anpd_status anpd_ngram_create(const anpd_ngram_config* cfg, void* cuda_stream, anpd_ngram** out);
@@ -190,6 +202,18 @@ anpd_status anpd_verify_batch(anpd_model* m, anpd_kv* kv, const int32_t* last_to
  * logits_host [(draft_len+1) * vocab] fp32; the cache length is left unchanged. */
 anpd_status anpd_verify_logits(anpd_model* m, anpd_kv* kv, int32_t last_tok, const int32_t* draft,
                                int draft_len, float* logits_host);
+
+/* Verification of two candidates in one step (the Conclusion's outlook: several candidates verified in parallel), for a
+ * kv handle of batch 1, the candidates brought by the host: draft_a [len_a] and draft_b [len_b], len_a >= 1, len_b >= 1,
+ * len_a + len_b <= ANPD_K_MAX (else ANPD_ERR_RANGE).  One forward over rows {last_tok, draft_a, draft_b}: the rows of
+ * draft_b take the positions right after last_tok again and attend to the committed context, last_tok and themselves,
+ * not to draft_a.  Each candidate's accepted prefix is found as in anpd_verify; the longer one is committed (draft_a on a
+ * tie): *chosen = 0 or 1, *accepted_len its accepted length, *next_tok the model's token after it, cache length =
+ * kv_len + accepted_len + 1, and the cache holds the chosen candidate's rows at their positions.  logits_host: NULL, or
+ * host memory for the (1 + len_a + len_b) * vocab fp32 logits of the rows in the order above (parity hook). */
+anpd_status anpd_verify_two_candidates(anpd_model* m, anpd_kv* kv, int32_t last_tok, const int32_t* draft_a, int len_a,
+                                       const int32_t* draft_b, int len_b, int* accepted_len, int32_t* next_tok,
+                                       int* chosen, float* logits_host);
 
 /* Asynchronous layer under anpd_verify_batch, for timing with events on the model's stream:
  * stage copies the step's inputs for all sequences to the device; enqueue issues the forward,

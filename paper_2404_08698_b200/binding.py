@@ -43,12 +43,12 @@ class NgramEntry(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("steps", C.c_int), ("drafted", C.c_int), ("accepted", C.c_int), ("generated", C.c_int),
-                ("hist_accepted", C.c_int * 8), ("ms_prefill", C.c_double), ("ms_decode", C.c_double),
+                ("hist_accepted", C.c_int * 8), ("alt_wins", C.c_int), ("reserved", C.c_int), ("ms_prefill", C.c_double), ("ms_decode", C.c_double),
                 ("bytes_per_step", C.c_double)]
 
     def as_dict(self) -> dict:
         return {"steps": self.steps, "drafted": self.drafted, "accepted": self.accepted, "generated": self.generated,
-                "hist_accepted": list(self.hist_accepted), "ms_prefill": self.ms_prefill, "ms_decode": self.ms_decode,
+                "hist_accepted": list(self.hist_accepted), "alt_wins": self.alt_wins, "ms_prefill": self.ms_prefill, "ms_decode": self.ms_decode,
                 "bytes_per_step": self.bytes_per_step}
 
 
@@ -70,6 +70,7 @@ SIGNATURES = {
     "anpd_kv_destroy": (C.c_int, [_P]),
     "anpd_kv_len": (C.c_int, [_P, C.c_int, _IP]),
     "anpd_kv_truncate": (C.c_int, [_P, C.c_int, C.c_int]),
+    "anpd_kv_set_candidates": (C.c_int, [_P, C.c_int]),
     "anpd_ngram_create": (C.c_int, [C.POINTER(NgramConfig), _P, C.POINTER(_P)]),
     "anpd_ngram_reset": (C.c_int, [_P]),
     "anpd_ngram_destroy": (C.c_int, [_P]),
@@ -82,6 +83,7 @@ SIGNATURES = {
     "anpd_verify": (C.c_int, [_P, _P, C.c_int32, _I32P, C.c_int, _IP, _I32P]),
     "anpd_verify_batch": (C.c_int, [_P, _P, _I32P, _I32P, _IP, _IP, _I32P]),
     "anpd_verify_logits": (C.c_int, [_P, _P, C.c_int32, _I32P, C.c_int, C.POINTER(C.c_float)]),
+    "anpd_verify_two_candidates": (C.c_int, [_P, _P, C.c_int32, _I32P, C.c_int, _I32P, C.c_int, _IP, _I32P, _IP, C.POINTER(C.c_float)]),
     "anpd_verify_stage": (C.c_int, [_P, _P, _I32P, _I32P, _IP]),
     "anpd_verify_enqueue": (C.c_int, [_P, _P]),
     "anpd_verify_result": (C.c_int, [_P, _P, _IP, _I32P]),
@@ -178,6 +180,10 @@ def anpd_kv_truncate(kv: int, seq: int, length: int) -> None:
     _check(lib().anpd_kv_truncate(_P(kv), seq, length), "anpd_kv_truncate")
 
 
+def anpd_kv_set_candidates(kv: int, candidates: int) -> None:
+    _check(lib().anpd_kv_set_candidates(_P(kv), candidates), "anpd_kv_set_candidates")
+
+
 # ---- n-gram ---------------------------------------------------------------------------------
 def anpd_ngram_create(n_min: int, n_max: int, max_ctx: int, policy: int = 0, stream: int = 0) -> int:
     cfg = NgramConfig(n_min, n_max, max_ctx, policy)
@@ -270,6 +276,18 @@ def anpd_verify_logits(m: int, kv: int, last_tok: int, draft, vocab: int) -> np.
     _check(lib().anpd_verify_logits(_P(m), _P(kv), int(last_tok), _ptr(d) if d.size else None, d.size,
                                     out.ctypes.data_as(C.POINTER(C.c_float))), "anpd_verify_logits")
     return out
+
+
+def anpd_verify_two_candidates(m: int, kv: int, last_tok: int, draft_a, draft_b, vocab: int = 0):
+    """(chosen, accepted_len, next_tok, logits or None); logits [(1 + len_a + len_b), vocab] when vocab > 0."""
+    a, b = _i32(draft_a), _i32(draft_b)
+    acc, nxt, chosen = C.c_int(), C.c_int32(), C.c_int()
+    out = np.zeros((1 + a.size + b.size, vocab), dtype=np.float32) if vocab > 0 else None
+    _check(lib().anpd_verify_two_candidates(_P(m), _P(kv), int(last_tok), _ptr(a) if a.size else None, a.size,
+                                            _ptr(b) if b.size else None, b.size, C.byref(acc), C.byref(nxt), C.byref(chosen),
+                                            out.ctypes.data_as(C.POINTER(C.c_float)) if out is not None else None),
+           "anpd_verify_two_candidates")
+    return chosen.value, acc.value, nxt.value, out
 
 
 def anpd_verify_stage(m: int, kv: int, last_tok, drafts) -> None:

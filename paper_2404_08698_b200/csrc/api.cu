@@ -65,6 +65,7 @@ __global__ void set_int_kernel(int* p, int v) { *p = v; }
 __global__ void seq_restart_kernel(SeqState* s) {
     s->kv_len = 0; s->draft_len = 0; s->accepted_len = 0;
     s->steps = 0; s->drafted = 0; s->accepted = 0;
+    s->draft2_len = 0; s->alt_wins = 0; s->move_n = 0;
     for (int i = 0; i < 8; ++i) s->hist[i] = 0;
     s->active = 1; s->stop_at = 0x7fffffff; s->error = 0;
 }
@@ -74,6 +75,7 @@ __global__ void greedy_stage_kernel(SeqState* seqs) {
     SeqState& s = seqs[blockIdx.x];
     s.last_tok = s.next_tok;
     s.draft_len = 0;
+    s.draft2_len = 0;
 }
 
 // Last kernel of a step inside the device-resident decoding loop: the loop goes on while a sequence is still active and
@@ -363,6 +365,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
     kv->max_len = kv->pages_per_seq * KV_PAGE;
     kv->total_pages = kv->pages_per_seq * batch;
     kv->staged = false;
+    kv->candidates = 1;
     kv->warm = false;
     kv->loop_ok = std::getenv("ANPD_HOST_LOOP") == nullptr;
     kv->side_stream = nullptr; kv->ev_fork = nullptr; kv->ev_join = nullptr;
@@ -397,6 +400,7 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
         {(void**)&kv->seq, sizeof(SeqState) * (size_t)batch}, {(void**)&kv->d_prompt, (size_t)kv->max_len * 4},
         {(void**)&kv->d_ctxs, sizeof(NgramDev) * (size_t)batch},
         {(void**)&ws.row_tok, R * 4}, {(void**)&ws.row_pos, R * 4}, {(void**)&ws.row_seq, R * 4}, {(void**)&ws.row_ok, R * 4},
+        {(void**)&ws.row_slot, R * 4}, {(void**)&ws.row_hole_lo, R * 4}, {(void**)&ws.row_hole_hi, R * 4},
         {(void**)&ws.x, R * d * 4}, {(void**)&ws.h_hi, R * d * 2}, {(void**)&ws.h_lo, R * d * 2},
         {(void**)&ws.ao_hi, R * m->dq * 2}, {(void**)&ws.ao_lo, R * m->dq * 2},
         {(void**)&ws.act_hi, R * F * 2}, {(void**)&ws.act_lo, R * F * 2},
@@ -628,13 +632,16 @@ anpd_status anpd_verify_stage(anpd_model* m, anpd_kv* kv, const int32_t* last_to
 // (the confirmed token alone); K < 0: the step's inputs were staged by the host.  Then the forward over
 // the batch * 8 rows, argmax / accept and, in COMMIT mode, the KV commit and token-buffer append.
 // Steps of one shape are captured once into a CUDA graph and replayed.
-static anpd_status step_enqueue(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K, int max_pos) {
+static anpd_status step_enqueue(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K, int max_pos, bool two) {
     cudaStream_t st = m->stream;
-    if (K > 0) ANPD_TRY(ngram_enqueue_step(d_ctxs, kv->seq, kv->batch, K, st, &m->prof));
+    // Two candidates per step (the Conclusion's outlook on verifying several candidates at once): the first keeps up to 4
+    // draft tokens, the alternative up to 3, so that both fit the step's 7 draft rows.
+    // (`two`; a host-staged step, K < 0, brings both candidates itself.)
+    if (K > 0) ANPD_TRY(ngram_enqueue_step(d_ctxs, kv->seq, kv->batch, two ? std::min(K, 4) : K, st, &m->prof, two ? std::min(K, 3) : 0));
     else if (K == 0) { LAUNCH(&m->prof, st, KC_OTHER, 0, (launch_k(greedy_stage_kernel, kv->batch, 1, 0, st, kv->seq))); }
-    ANPD_TRY(plan_decode_enqueue(m, kv));
-    ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits));
-    ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0));
+    ANPD_TRY(plan_decode_enqueue(m, kv, two));
+    ANPD_TRY(forward_enqueue(m, kv, kv->batch * ANPD_ROWS, max_pos, true, want_logits, 0, two));
+    ANPD_TRY(accept_enqueue(m, kv, mode, d_ctxs, 0, 0, 0, two));
     return ANPD_OK;
 }
 
@@ -646,7 +653,8 @@ static anpd_status step_enqueue(anpd_model* m, anpd_kv* kv, int mode, bool want_
 static anpd_status decode_loop_enqueue(anpd_model* m, anpd_kv* kv, const NgramDev* d_ctxs, int K, int max_pos_bound, int max_steps) {
     if (!kv->use_graphs || m->prof.on || !kv->loop_ok) return ANPD_ERR_STATE;
     cudaStream_t st = m->stream;
-    const uint64_t key = (uint64_t)(max_pos_bound / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)(d_ctxs ? 1 : 0) << 29);
+    const uint64_t key = (uint64_t)(max_pos_bound / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)(d_ctxs ? 1 : 0) << 29) |
+                         ((uint64_t)(kv->candidates == 2 ? 1 : 0) << 30);
     auto it = kv->loop_graphs.find(key);
     if (it == kv->loop_graphs.end()) {
         if (!kv->warm) {                                // one eager step first: function attributes, lazy module loading
@@ -671,7 +679,7 @@ static anpd_status decode_loop_enqueue(anpd_model* m, anpd_kv* kv, const NgramDe
             const long long before = g_launch_count.load();
             ok = cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
             if (ok) {
-                anpd_status rc = step_enqueue(m, kv, ACCEPT_COMMIT, false, d_ctxs, K, max_pos_bound);
+                anpd_status rc = step_enqueue(m, kv, ACCEPT_COMMIT, false, d_ctxs, K, max_pos_bound, K > 0 && kv->candidates == 2);
                 if (rc == ANPD_OK) {
                     LAUNCH(&m->prof, st, KC_OTHER, 0,
                            (launch_k(loop_condition_kernel, 1, 32, 0, st, kv->seq, kv->batch, kv->ws.gemm_err, kv->loop_steps_left, handle)));
@@ -701,7 +709,7 @@ static anpd_status decode_loop_enqueue(anpd_model* m, anpd_kv* kv, const NgramDe
     return ANPD_OK;
 }
 
-static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K = -1) {
+static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, bool want_logits, const NgramDev* d_ctxs, int K = -1, bool two = false) {
     ANPD_TRY(check_device(m));
     int max_pos = 0;
     for (int b = 0; b < kv->batch; ++b) {
@@ -711,7 +719,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
         max_pos = std::max(max_pos, kv->h_kv_len[b] + ANPD_ROWS - 1);
     }
     cudaStream_t st = m->stream;
-    auto enqueue = [&]() -> anpd_status { return step_enqueue(m, kv, mode, want_logits, d_ctxs, K, max_pos); };
+    auto enqueue = [&]() -> anpd_status { return step_enqueue(m, kv, mode, want_logits, d_ctxs, K, max_pos, two); };
     if (m->prof.on || !kv->use_graphs || !kv->warm) {
         kv->warm = true;
         NoPdlScope no_overlap(m->prof.on);            // per-launch timing needs kernels that do not overlap
@@ -720,7 +728,7 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
         return rc;
     }
     const uint64_t key = (uint64_t)(max_pos / KV_PAGE) | ((uint64_t)(K + 1) << 16) | ((uint64_t)mode << 24) |
-                         ((uint64_t)(want_logits ? 1 : 0) << 28) | ((uint64_t)(d_ctxs ? 1 : 0) << 29);
+                         ((uint64_t)(want_logits ? 1 : 0) << 28) | ((uint64_t)(d_ctxs ? 1 : 0) << 29) | ((uint64_t)(two ? 1 : 0) << 30);
     auto it = kv->graphs.find(key);
     if (it == kv->graphs.end()) {
         const long long before = g_launch_count.load();
@@ -747,6 +755,13 @@ static anpd_status verify_enqueue_mode(anpd_model* m, anpd_kv* kv, int mode, boo
     CUDA_TRY(cudaGraphLaunch(it->second.exec, st));
     g_launch_count += it->second.launches;
     if (mode == ACCEPT_COMMIT) std::fill(kv->h_len_stale.begin(), kv->h_len_stale.end(), 1);
+    return ANPD_OK;
+}
+
+anpd_status anpd_kv_set_candidates(anpd_kv* kv, int candidates) {
+    if (!kv) return ANPD_ERR_ARG;
+    if (candidates != 1 && candidates != 2) return ANPD_ERR_RANGE;
+    kv->candidates = candidates;
     return ANPD_OK;
 }
 
@@ -795,6 +810,33 @@ anpd_status anpd_verify_logits(anpd_model* m, anpd_kv* kv, int32_t last_tok, con
                              cudaMemcpyDeviceToHost, m->stream));
     ANPD_TRY(read_seqs(kv));
     return seq_error_status(kv->h_seq[0]);
+}
+
+anpd_status anpd_verify_two_candidates(anpd_model* m, anpd_kv* kv, int32_t last_tok, const int32_t* draft_a, int len_a,
+                                       const int32_t* draft_b, int len_b, int* accepted_len, int32_t* next_tok, int* chosen,
+                                       float* logits_host) {
+    if (!m || !kv || kv->m != m || kv->batch != 1 || !accepted_len || !next_tok || !chosen || !draft_a || !draft_b) return ANPD_ERR_ARG;
+    if (len_a < 1 || len_b < 1 || len_a + len_b > ANPD_K_MAX) return ANPD_ERR_RANGE;
+    for (int i = 0; i < len_b; ++i)
+        if (draft_b[i] < 0 || draft_b[i] >= m->cfg.vocab) return ANPD_ERR_RANGE;
+    int32_t padded[ANPD_K_MAX] = {0};
+    for (int i = 0; i < len_a; ++i) padded[i] = draft_a[i];
+    ANPD_TRY(anpd_verify_stage(m, kv, &last_tok, padded, &len_a));
+    // draft2_len and draft2[] are adjacent in SeqState too
+    int* stage = kv->h_small + (2 + ANPD_K_MAX + 1);
+    stage[0] = len_b;
+    for (int i = 0; i <= ANPD_K_MAX; ++i) stage[1 + i] = (i < len_b) ? draft_b[i] : 0;
+    CUDA_TRY(cudaMemcpyAsync(&kv->seq[0].draft2_len, stage, (2 + ANPD_K_MAX) * sizeof(int), cudaMemcpyHostToDevice, m->stream));
+    ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, logits_host != nullptr, nullptr, -1, true));
+    if (logits_host)
+        CUDA_TRY(cudaMemcpyAsync(logits_host, kv->ws.logits, sizeof(float) * (size_t)(len_a + len_b + 1) * m->cfg.vocab,
+                                 cudaMemcpyDeviceToHost, m->stream));
+    ANPD_TRY(read_seqs(kv));
+    ANPD_TRY(seq_error_status(kv->h_seq[0]));
+    *accepted_len = kv->h_seq[0].accepted_len;
+    *next_tok = kv->h_seq[0].next_tok;
+    *chosen = kv->h_seq[0].move_n > 0 ? 1 : 0;
+    return ANPD_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -863,7 +905,7 @@ static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* 
             const anpd_status lrc = decode_loop_enqueue(m, kv, kv->d_ctxs, K, max_pos_bound, max_new + 2);
             if (lrc == ANPD_OK) g_launch_count += 0;    // counted below from the steps the sequences report
             else if (lrc != ANPD_ERR_STATE) return lrc;
-            else ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs, K));
+            else ANPD_TRY(verify_enqueue_mode(m, kv, ACCEPT_COMMIT, false, kv->d_ctxs, K, K > 0 && kv->candidates == 2));
             int steps_before = 0;
             for (int b = 0; b < B; ++b) steps_before = std::max(steps_before, kv->h_seq[b].steps);
             ANPD_TRY(read_seqs(kv));
@@ -898,6 +940,7 @@ static anpd_status generate_core(anpd_model* m, anpd_kv* kv, anpd_ngram* const* 
                 anpd_stats& o = stats[b];
                 o.steps = s.steps; o.drafted = s.drafted; o.accepted = s.accepted; o.generated = nt - prompt_len - 1;
                 for (int i = 0; i < 8; ++i) o.hist_accepted[i] = s.hist[i];
+                o.alt_wins = s.alt_wins; o.reserved = 0;
                 o.ms_prefill = ms_p; o.ms_decode = ms_d;
                 const double mean_kv = prompt_len + 0.5 * (nt - prompt_len - 1);
                 const anpd_model_config& c = m->cfg;

@@ -75,7 +75,10 @@ __global__ void __launch_bounds__(AttnCfg<G, S>::THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const bf16* __restrict__ q_hi,
                const bf16* __restrict__ q_lo, const int* __restrict__ page_table, int pages_per_seq, const int* __restrict__ row_pos,
                const int* __restrict__ row_seq, int Hq, int Hkv, int layer_row0, int chunks, int n_items, float* __restrict__ pm,
-               float* __restrict__ pl, float* __restrict__ po, int* err) {
+               float* __restrict__ pl, float* __restrict__ po, int* err, const int* __restrict__ row_slot,
+               const int* __restrict__ row_hole_lo, const int* __restrict__ row_hole_hi) {
+    // row_slot / row_hole_*: null except in two-candidate steps, where row r of a group lives in cache slot pos_lo + r, its
+    // group reaches up to row_slot[last row], and a second candidate's rows must not see the slots [hole_lo, hole_hi)
     typedef AttnCfg<G, S> Cfg;
     constexpr int Q = Cfg::Q, N = Cfg::N, SLOTS = Cfg::SLOTS;
     extern __shared__ __align__(1024) unsigned char attn_tc_smem[];
@@ -123,7 +126,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
     auto next_item = [&](int it, AttnItem& out) -> int {
         for (; it < n_items; it += stride) {
             decode(it, out);
-            const int hi = row_pos[out.r0 + ANPD_ROWS - 1];          // three independent loads
+            const int hi = (row_slot ? row_slot : row_pos)[out.r0 + ANPD_ROWS - 1];          // three independent loads
             out.pos_lo = row_pos[out.r0];
             out.seq = row_seq[out.r0];
             if (out.c * KV_PAGE <= hi) return it;
@@ -216,6 +219,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
             if (key > cur.pos_lo + (q & 7)) s[q] = -CUDART_INF_F;
+            if (row_slot && key >= row_hole_lo[cur.r0 + (q & 7)] && key < row_hole_hi[cur.r0 + (q & 7)]) s[q] = -CUDART_INF_F;
             float mx = s[q];
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
             if (lane == 0) red_max[slot][warp][q] = mx;
@@ -497,7 +501,7 @@ attn_prompt_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 }
 
 template <int G, int S>
-anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int chunks) {
+anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int chunks, bool tree) {
     typedef AttnCfg<G, S> Cfg;
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
@@ -511,7 +515,8 @@ anpd_status launch_attn_tc(anpd_model* m, anpd_kv* kv, int layer, int rows, int 
     LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (launch_k(attn_tc_kernel<G, S>, grid, Cfg::THREADS, Cfg::SMEM, m->stream, kv->map_k, kv->map_v, ws.q_hi, ws.q_lo, kv->page_table,
                      kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads, c.n_kv_heads, layer_row0, chunks, n_items, ws.attn_m,
-                     ws.attn_l, ws.attn_o, ws.gemm_err)));
+                     ws.attn_l, ws.attn_o, ws.gemm_err, tree ? ws.row_slot : (const int*)nullptr,
+                     tree ? ws.row_hole_lo : (const int*)nullptr, tree ? ws.row_hole_hi : (const int*)nullptr)));
     return ANPD_OK;
 }
 
@@ -536,17 +541,17 @@ anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows)
     return ANPD_OK;
 }
 
-anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos) {
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool tree) {
     const int chunks = max_pos / KV_PAGE + 1;
     const int n_items = chunks * m->cfg.n_kv_heads * (rows / ANPD_ROWS);
     switch (m->cfg.n_q_heads / m->cfg.n_kv_heads) {
         // one query head per kv head fits five slots; while every item finds a slot with four, four are faster
         // (measured at the 7B shape: 1.2 % of the step at 17 pages; with 33 pages five slots win by 2.4 %)
-        case 1: return n_items <= 4 * m->num_sms ? launch_attn_tc<1, 4>(m, kv, layer, rows, chunks)
-                                                 : launch_attn_tc<1, 5>(m, kv, layer, rows, chunks);
-        case 2: return launch_attn_tc<2, 4>(m, kv, layer, rows, chunks);
-        case 4: return launch_attn_tc<4, 3>(m, kv, layer, rows, chunks);
-        case 8: return launch_attn_tc<8, 2>(m, kv, layer, rows, chunks);
+        case 1: return n_items <= 4 * m->num_sms ? launch_attn_tc<1, 4>(m, kv, layer, rows, chunks, tree)
+                                                 : launch_attn_tc<1, 5>(m, kv, layer, rows, chunks, tree);
+        case 2: return launch_attn_tc<2, 4>(m, kv, layer, rows, chunks, tree);
+        case 4: return launch_attn_tc<4, 3>(m, kv, layer, rows, chunks, tree);
+        case 8: return launch_attn_tc<8, 2>(m, kv, layer, rows, chunks, tree);
     }
     return ANPD_ERR_ARG;
 }

@@ -26,26 +26,35 @@ __device__ __forceinline__ void split_bf16(float v, bf16& hi, bf16& lo) {
 // ---------------------------------------------------------------------------------------------
 // row plans
 // ---------------------------------------------------------------------------------------------
-__global__ void plan_decode_kernel(SeqState* seqs, int* row_tok, int* row_pos, int* row_seq, int* row_ok,
-                                   int vocab, int max_len) {
+// Rows of a sequence's step: row 0 the confirmed token at position P; rows 1..ka the first candidate at positions P+1..;
+// with a second candidate (two-candidate mode) rows ka+1..ka+kb hold its tokens at positions P+1.. again, but their K/V go
+// to the cache slots behind the first candidate's (slot = P + row), and they must not see the first candidate's slots.
+__global__ void plan_decode_kernel(SeqState* seqs, int* row_tok, int* row_pos, int* row_seq, int* row_ok, int* row_slot,
+                                   int* row_hole_lo, int* row_hole_hi, int vocab, int max_len, int two) {
     pdl_trigger();
     pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int b = i / ANPD_ROWS, r = i % ANPD_ROWS;
     SeqState& s = seqs[b];
-    int tok = (r == 0) ? s.last_tok : (r <= s.draft_len ? s.draft[r - 1] : 0);
-    if (tok < 0 || tok >= vocab) { if (r <= s.draft_len) atomicExch(&s.error, ERR_TOKEN_RANGE); tok = 0; }
-    const int pos = s.kv_len + r;
-    if (pos >= max_len && r <= s.draft_len && s.active) atomicExch(&s.error, ERR_KV_FULL);
+    const int ka = s.draft_len, kb = two ? min(s.draft2_len, ANPD_K_MAX - ka) : 0;
+    const bool real = r <= ka + kb;
+    int tok = (r == 0) ? s.last_tok : (r <= ka ? s.draft[r - 1] : (real ? s.draft2[r - ka - 1] : 0));
+    if (tok < 0 || tok >= vocab) { if (real) atomicExch(&s.error, ERR_TOKEN_RANGE); tok = 0; }
+    const int slot = s.kv_len + r;
+    const int pos = (r > ka && real) ? s.kv_len + (r - ka) : slot;
+    if (slot >= max_len && real && s.active) atomicExch(&s.error, ERR_KV_FULL);
     row_tok[i] = tok;
     row_pos[i] = min(pos, max_len - 1);
     row_seq[i] = b;
-    row_ok[i] = (pos < max_len) ? 1 : 0;
+    row_ok[i] = (slot < max_len) ? 1 : 0;
+    row_slot[i] = min(slot, max_len - 1);
+    row_hole_lo[i] = (r > ka && real) ? s.kv_len + 1 : 0;
+    row_hole_hi[i] = (r > ka && real) ? s.kv_len + ka + 1 : 0;
 }
 
 __global__ void plan_prefill_kernel(const int* prompt, int seq, int start, int prompt_len, int rows,
-                                    int* row_tok, int* row_pos, int* row_seq, int* row_ok, int vocab, int max_len,
-                                    SeqState* seqs) {
+                                    int* row_tok, int* row_pos, int* row_seq, int* row_ok, int* row_slot, int* row_hole_lo,
+                                    int* row_hole_hi, int vocab, int max_len, SeqState* seqs) {
     pdl_trigger();
     pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -57,6 +66,9 @@ __global__ void plan_prefill_kernel(const int* prompt, int seq, int start, int p
     row_pos[i] = min(p, max_len - 1);
     row_seq[i] = seq;
     row_ok[i] = (p < max_len && p < prompt_len) ? 1 : 0;
+    row_slot[i] = min(p, max_len - 1);
+    row_hole_lo[i] = 0;
+    row_hole_hi[i] = 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -196,7 +208,7 @@ __global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restr
 // QKV epilogue: reduce splits, rotary embedding, append K/V to the paged cache, keep q
 // ---------------------------------------------------------------------------------------------
 __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride, int ld_part,
-                                       const int* __restrict__ row_pos, const int* __restrict__ row_seq,
+                                       const int* __restrict__ row_pos, const int* __restrict__ row_slot, const int* __restrict__ row_seq,
                                        const int* __restrict__ row_ok, const float* __restrict__ rope_cos,
                                        const float* __restrict__ rope_sin, const int* __restrict__ page_table,
                                        int pages_per_seq, int Hq, int Hkv, int hd, float q_scale, bf16* __restrict__ q_hi,
@@ -227,14 +239,15 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
     if (!row_ok[row]) return;
     const bool is_k = head < Hq + Hkv;
     const int kvh = is_k ? head - Hq : head - Hq - Hkv;
-    const int page = page_table[row_seq[row] * pages_per_seq + pos / KV_PAGE];
+    const int slot = row_slot[row];               // where the row lives in the cache (its position, except for a second candidate)
+    const int page = page_table[row_seq[row] * pages_per_seq + slot / KV_PAGE];
     bf16* pg = (is_k ? kpool_l : vpool_l) + ((size_t)page * Hkv + kvh) * KV_PAGE * hd;
     if (is_k) {                                   // K page: [position][dim]
-        pg[(size_t)(pos % KV_PAGE) * hd + i] = __float2bfloat16_rn(a);
-        pg[(size_t)(pos % KV_PAGE) * hd + i + half] = __float2bfloat16_rn(b);
+        pg[(size_t)(slot % KV_PAGE) * hd + i] = __float2bfloat16_rn(a);
+        pg[(size_t)(slot % KV_PAGE) * hd + i + half] = __float2bfloat16_rn(b);
     } else {                                      // V page is kept transposed: [dim][position]
-        pg[(size_t)i * KV_PAGE + (pos % KV_PAGE)] = __float2bfloat16_rn(a);
-        pg[(size_t)(i + half) * KV_PAGE + (pos % KV_PAGE)] = __float2bfloat16_rn(b);
+        pg[(size_t)i * KV_PAGE + (slot % KV_PAGE)] = __float2bfloat16_rn(a);
+        pg[(size_t)(i + half) * KV_PAGE + (slot % KV_PAGE)] = __float2bfloat16_rn(b);
     }
 }
 
@@ -361,7 +374,8 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const bf16* 
                                                                     const int* __restrict__ page_table, int pages_per_seq,
                                                                     const int* __restrict__ row_pos, const int* __restrict__ row_seq, int Hq,
                                                                     int Hkv, float* __restrict__ pm, float* __restrict__ pl,
-                                                                    float* __restrict__ po) {
+                                                                    float* __restrict__ po, const int* __restrict__ row_slot,
+                                                                    const int* __restrict__ row_hole_lo, const int* __restrict__ row_hole_hi) {
     pdl_trigger();
     pdl_wait();
     constexpr int SLABS = HD / 32;            // 32-wide slabs of the head dimension (two MMAs each)
@@ -379,7 +393,8 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const bf16* 
     const int MT = (ANPD_ROWS * G + 15) / 16;             // 16-row tiles of query vectors: 1, 1, 2, 4 for G = 1, 2, 4, 8
     const int KG = 4 / MT;                                // warps that split the page's four key blocks
     const int c = blockIdx.x, kvh = blockIdx.y, r0 = blockIdx.z * ANPD_ROWS;
-    const int pos_lo = row_pos[r0], pos_hi = row_pos[r0 + ANPD_ROWS - 1];
+    // row_slot (two-candidate steps): a row sees the cache slots up to its own, except a hidden range; otherwise slot = position
+    const int pos_lo = row_pos[r0], pos_hi = row_slot ? row_slot[r0 + ANPD_ROWS - 1] : row_pos[r0 + ANPD_ROWS - 1];
     if (c * KV_PAGE > pos_hi) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, t = lane & 3;
     const int mt = warp % MT, kg = warp / MT;
@@ -406,14 +421,15 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const bf16* 
     }
 
     // this thread's two query vectors (rows gid and gid + 8 of tile mt) and their positions
-    int qpos[2];
+    int qpos[2], qhl[2] = {0, 0}, qhh[2] = {0, 0};
     uint32_t qh[SLABS][2][4], ql[SLABS][2][4];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const int qi = mt * 16 + gid + 8 * h;
         const bool valid = qi < ANPD_ROWS * G;
         const int r = valid ? qi / G : 0, hl = valid ? qi % G : 0;
-        qpos[h] = valid ? pos_lo + r : -1;                // -1: padding row, sees no key
+        qpos[h] = valid ? (row_slot ? row_slot[r0 + r] : pos_lo + r) : -1;                // -1: padding row, sees no key
+        if (valid && row_slot) { qhl[h] = row_hole_lo[r0 + r]; qhh[h] = row_hole_hi[r0 + r]; }
         const size_t qoff = (size_t)(r0 + r) * Hq * HD + (size_t)(kvh * G + hl) * HD + 8 * t;
 #pragma unroll
         for (int s = 0; s < SLABS; ++s) {
@@ -461,7 +477,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_partial_kernel(const bf16* 
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int key = kb0 + 8 * t + 2 * j + e;
-                    const float v = (key <= qpos[h]) ? sc[j][2 * h + e] : -CUDART_INF_F;
+                    const float v = (key <= qpos[h] && !(key >= qhl[h] && key < qhh[h])) ? sc[j][2 * h + e] : -CUDART_INF_F;
                     sc[j][2 * h + e] = v;
                     mx = fmaxf(mx, v);
                 }
@@ -564,6 +580,7 @@ constexpr int COMBINE_MAX_PAGES = 256;
 __global__ void attn_combine_kernel(const float* __restrict__ pm, const float* __restrict__ pl, const float* __restrict__ po,
                                     const int* __restrict__ row_pos, int Hq, int hd, int pages_per_seq,
                                     bf16* __restrict__ ao_hi, bf16* __restrict__ ao_lo, unsigned char* __restrict__ img) {
+    // row_pos: the rows' cache slots (= positions outside two-candidate steps)
     pdl_trigger();
     pdl_wait();
     __shared__ float s_w[COMBINE_MAX_PAGES];            // page maxima, then page weights
@@ -756,7 +773,7 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const float* __rest
 // Final argmax per row, draft compare, prefix accept, KV commit, token-buffer append.
 __global__ void __launch_bounds__(256) accept_kernel(SeqState* seqs, const float* __restrict__ amax_val,
                                                      const int* __restrict__ amax_idx, int nblk, int mode,
-                                                     const NgramDev* ctxs, int seq_arg, int last_row, int prompt_len) {
+                                                     const NgramDev* ctxs, int seq_arg, int last_row, int prompt_len, int two) {
     pdl_trigger();
     pdl_wait();
     __shared__ int pred[ANPD_ROWS];
@@ -796,24 +813,66 @@ __global__ void __launch_bounds__(256) accept_kernel(SeqState* seqs, const float
         return;
     }
     int a = 0;
-    while (a < s.draft_len && s.draft[a] == pred[a]) ++a;
+    const int ka = s.draft_len;
+    while (a < ka && s.draft[a] == pred[a]) ++a;
     for (int r = 0; r < ANPD_ROWS; ++r) s.pred[r] = pred[r];
+    // A second candidate (rows ka+1..ka+kb): its first token is judged by row 0's prediction, token j by the prediction of
+    // its own row before (row ka+j).  It is kept when its accepted prefix is strictly longer; the first candidate wins ties.
+    const int kb = two ? min(s.draft2_len, ANPD_K_MAX - ka) : 0;
+    const int* chosen = s.draft;
+    int nxt = pred[a];
+    if (two) s.move_n = 0;
+    if (kb > 0 && s.draft2[0] == pred[0]) {
+        int ab = 1;
+        while (ab < kb && s.draft2[ab] == pred[ka + ab]) ++ab;
+        if (ab > a) {
+            chosen = s.draft2;
+            a = ab;
+            nxt = pred[ka + ab];
+            if (mode == ACCEPT_COMMIT && s.active) {           // its K/V rows sit behind the first candidate's: ask for the move
+                s.move_from = s.kv_len + ka + 1;
+                s.move_to = s.kv_len + 1;
+                s.move_n = ab;
+                s.alt_wins += 1;
+            }
+        }
+    }
     s.accepted_len = a;
-    s.next_tok = pred[a];
+    s.next_tok = nxt;
     if (mode != ACCEPT_COMMIT || !s.active) return;
     s.kv_len += a + 1;
     s.steps += 1;
-    s.drafted += s.draft_len;
+    s.drafted += ka + kb;
     s.accepted += a;
     s.hist[a] += 1;
     if (ctxs) {
         const NgramDev& c = ctxs[b];
         const int T = c.state[0];
         if (T + a + 1 > c.max_ctx) { s.error = ERR_CTX_FULL; s.active = 0; return; }
-        for (int i = 0; i < a; ++i) c.tokens[T + i] = s.draft[i];
-        c.tokens[T + a] = pred[a];
+        for (int i = 0; i < a; ++i) c.tokens[T + i] = chosen[i];
+        c.tokens[T + a] = nxt;
         c.state[0] = T + a + 1;
         if (T + a + 1 >= s.stop_at) s.active = 0;
+    }
+}
+
+// Two-candidate steps: when the second candidate won, its accepted rows' K and V move from the slots behind the first
+// candidate's to the positions they belong to (SeqState::move_*).  One thread per (layer, kv head, dim) walks the rows in
+// ascending order, so overlapping ranges behave like memmove.  grid (layers * kv heads, batch), hd threads.
+__global__ void kv_move_kernel(const SeqState* __restrict__ seqs, const int* __restrict__ page_table, int pages_per_seq, int Hkv, int hd,
+                               size_t layer_elems, bf16* __restrict__ kpool, bf16* __restrict__ vpool) {
+    pdl_trigger();
+    pdl_wait();
+    const SeqState& s = seqs[blockIdx.y];
+    const int n = s.move_n;
+    if (n <= 0) return;
+    const int layer = blockIdx.x / Hkv, kvh = blockIdx.x % Hkv, i = threadIdx.x;
+    for (int j = 0; j < n; ++j) {
+        const int from = s.move_from + j, to = s.move_to + j;
+        const size_t pf = ((size_t)page_table[blockIdx.y * pages_per_seq + from / KV_PAGE] * Hkv + kvh) * KV_PAGE * hd + layer * layer_elems;
+        const size_t pt = ((size_t)page_table[blockIdx.y * pages_per_seq + to / KV_PAGE] * Hkv + kvh) * KV_PAGE * hd + layer * layer_elems;
+        kpool[pt + (size_t)(to % KV_PAGE) * hd + i] = kpool[pf + (size_t)(from % KV_PAGE) * hd + i];
+        vpool[pt + (size_t)i * KV_PAGE + (to % KV_PAGE)] = vpool[pf + (size_t)i * KV_PAGE + (from % KV_PAGE)];
     }
 }
 
@@ -904,7 +963,7 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
 }
 
 template <int HD>
-anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, unsigned char* img = nullptr) {
+anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, unsigned char* img = nullptr, bool tree = false) {
     const anpd_model_config& c = m->cfg;
     Workspace& ws = kv->ws;
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * HD;
@@ -918,19 +977,20 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && c.n_q_heads == c.n_kv_heads)
         return attn_prompt_enqueue(m, kv, layer, rows);          // a prompt pass: pages are folded in the kernel, nothing to merge
     if (HD == 128 && kv->attn_tc) {
-        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos));
+        ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos, tree));
     } else {
         dim3 grid(chunks, c.n_kv_heads, rows / ANPD_ROWS);
         LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
                (launch_k(attn_partial_kernel<HD>, grid, ATTN_THREADS, smem, m->stream, ws.q_hi, ws.q_lo, kv->kpool + layer * layer_elems,
                          kv->vpool + layer * layer_elems, kv->page_table, kv->pages_per_seq, ws.row_pos, ws.row_seq, c.n_q_heads,
-                         c.n_kv_heads, ws.attn_m, ws.attn_l, ws.attn_o)));
+                         c.n_kv_heads, ws.attn_m, ws.attn_l, ws.attn_o, tree ? ws.row_slot : (const int*)nullptr,
+                         tree ? ws.row_hole_lo : (const int*)nullptr, tree ? ws.row_hole_hi : (const int*)nullptr)));
     }
     if (rows >= 64) LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
            (launch_k(attn_combine_wide_kernel<HD / 32>, dim3(rows, c.n_q_heads), 32 * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o,
-                     ws.row_pos, c.n_q_heads, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
+                     tree ? ws.row_slot : ws.row_pos, c.n_q_heads, kv->pages_per_seq, ws.ao_hi, ws.ao_lo)));
     else LAUNCH(&m->prof, m->stream, KC_ATTN, 0,
-           (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, ws.row_pos, c.n_q_heads,
+           (launch_k(attn_combine_kernel, dim3(rows, c.n_q_heads), HD * COMBINE_SLICES, 0, m->stream, ws.attn_m, ws.attn_l, ws.attn_o, tree ? ws.row_slot : ws.row_pos, c.n_q_heads,
                                                                               HD, kv->pages_per_seq, ws.ao_hi, ws.ao_lo, img)));
     return ANPD_OK;
 }
@@ -946,11 +1006,12 @@ anpd_status gemm_plain_enqueue(const GemmPlan& p, const bf16* W, const bf16* a_h
     return ANPD_OK;
 }
 
-anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv) {
+anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv, bool two_candidates) {
     Workspace& ws = kv->ws;
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
            (launch_k(plan_decode_kernel, kv->batch, ANPD_ROWS, 0, m->stream, kv->seq, ws.row_tok, ws.row_pos, ws.row_seq, ws.row_ok,
-                                                                      m->cfg.vocab, kv->max_len)));
+                                                                      ws.row_slot, ws.row_hole_lo, ws.row_hole_hi, m->cfg.vocab, kv->max_len,
+                                                                      two_candidates ? 1 : 0)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
@@ -959,18 +1020,25 @@ anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start,
     Workspace& ws = kv->ws;
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
            (launch_k(plan_prefill_kernel, (rows + 127) / 128, 128, 0, m->stream, kv->d_prompt, seq, start, prompt_len, rows, ws.row_tok,
-                                                                          ws.row_pos, ws.row_seq, ws.row_ok, m->cfg.vocab,
-                                                                          kv->max_len, kv->seq)));
+                                                                          ws.row_pos, ws.row_seq, ws.row_ok, ws.row_slot, ws.row_hole_lo,
+                                                                          ws.row_hole_hi, m->cfg.vocab, kv->max_len, kv->seq)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
 
-anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len) {
+anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len, bool two_candidates) {
     Workspace& ws = kv->ws;
     const int blocks = (mode == ACCEPT_PREFILL) ? 1 : kv->batch;
     LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
            (launch_k(accept_kernel, blocks, 256, 0, m->stream, kv->seq, ws.amax_val_use, ws.amax_idx_use,
-                     ws.amax_nblk, mode, d_ctxs, seq, last_row, prompt_len)));
+                     ws.amax_nblk, mode, d_ctxs, seq, last_row, prompt_len, two_candidates ? 1 : 0)));
+    if (two_candidates && mode == ACCEPT_COMMIT) {
+        const anpd_model_config& c = m->cfg;
+        LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
+               (launch_k(kv_move_kernel, dim3(c.n_layers * c.n_kv_heads, kv->batch), c.head_dim, 0, m->stream, (const SeqState*)kv->seq,
+                         (const int*)kv->page_table, kv->pages_per_seq, c.n_kv_heads, c.head_dim,
+                         (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * c.head_dim, kv->kpool, kv->vpool)));
+    }
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }
@@ -1021,9 +1089,10 @@ static anpd_status forward_rr_enqueue(anpd_model* m, anpd_kv* kv, int max_pos, b
     return ANPD_OK;
 }
 
-anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits, int head_row) {
-    if (m->rr_ready && kv->batch == 1 && rows == ANPD_ROWS && head && !m->plain_gemm) return forward_rr_enqueue(m, kv, max_pos, want_logits);
-    if (kv->step_ready && rows == kv->batch * ANPD_ROWS && head && !m->prof.on) return step_kernel_enqueue(m, kv, max_pos, want_logits);
+anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits, int head_row, bool two_candidates) {
+    // the two fused variants know nothing of a second candidate's cache slots and mask
+    if (m->rr_ready && kv->batch == 1 && rows == ANPD_ROWS && head && !m->plain_gemm && !two_candidates) return forward_rr_enqueue(m, kv, max_pos, want_logits);
+    if (kv->step_ready && rows == kv->batch * ANPD_ROWS && head && !m->prof.on && !two_candidates) return step_kernel_enqueue(m, kv, max_pos, want_logits);
     const anpd_model_config& c = m->cfg;
     kv->ws.amax_nblk = kv->ws.amax_blocks;
     kv->ws.amax_val_use = kv->ws.amax_val;
@@ -1058,11 +1127,11 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
         } else
         LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(qkv_rope_append_kernel, dim3(rows, (c.n_q_heads + 2 * c.n_kv_heads + rope_hpb - 1) / rope_hpb), rope_hpb * (hd / 2), 0, st, 
-                   ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
+                   ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_slot, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
                    kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, hd, 1.4426950408889634f / sqrtf((float)hd), ws.q_hi,
                    ws.q_lo, kv->kpool + l * layer_elems, kv->vpool + l * layer_elems)));
-        if (hd == 128) ANPD_TRY(attn_enqueue<128>(m, kv, l, rows, max_pos));
-        else ANPD_TRY(attn_enqueue<64>(m, kv, l, rows, max_pos));
+        if (hd == 128) ANPD_TRY(attn_enqueue<128>(m, kv, l, rows, max_pos, nullptr, two_candidates));
+        else ANPD_TRY(attn_enqueue<64>(m, kv, l, rows, max_pos, nullptr, two_candidates));
         ANPD_TRY(gemm_enqueue(m, kv, GK_O, l, rows, &segs));
         LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(resid_norm_kernel, rows, NORM_THREADS, 0, st, ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,

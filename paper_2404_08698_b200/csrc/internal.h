@@ -126,6 +126,12 @@ struct SeqState {
     int active;                    // 0: the sequence idles (finished or out of room)
     int stop_at;                   // the loop retires the sequence once its context holds this many tokens
     int error;                     // sticky device-side error code
+    // a second candidate of the step (two-candidate mode): its tokens, how often it won, and the cache rows the accept
+    // step asks to be moved when it wins (its rows were written behind the first candidate's)
+    int draft2_len;
+    int draft2[ANPD_K_MAX + 1];
+    int alt_wins;
+    int move_from, move_to, move_n;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -169,8 +175,9 @@ struct anpd_ngram {
 anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof, cudaStream_t on = nullptr);
 // One fused launch for `batch` sequences: folds tokens [state[1], state[0]) of each, then drafts
 // K tokens into seq[b] (draft, draft_len, last_tok).
+// K2 > 0: also draft a second candidate of up to K2 tokens into seq[b].draft2
 anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batch, int K,
-                               cudaStream_t st, Profiler* prof);
+                               cudaStream_t st, Profiler* prof, int K2 = 0);
 
 // proj_rr.cu: the projections of a single-sequence step with their epilogues fused in ("row-range" kernel: each
 // CTA owns a contiguous range of output features and the whole contraction dimension).
@@ -282,6 +289,8 @@ struct Workspace {
     int n_max_out;                    // widest GEMM output (max of nqkv, 2F, d, V)
     int splits_max;
     int* row_tok; int* row_pos; int* row_seq; int* row_ok;    // [r_max]
+    // two-candidate mode: the cache slot a row's K/V go to (its position otherwise) and a range of slots it must not see
+    int* row_slot; int* row_hole_lo; int* row_hole_hi;          // [r_max]
     float* x;                         // [r_max, d] residual stream
     __nv_bfloat16 *h_hi, *h_lo;       // [r_max, d]   normalised input of QKV / gate-up / LM head
     __nv_bfloat16 *ao_hi, *ao_lo;     // [r_max, dq]  attention output, input of the O projection
@@ -364,6 +373,7 @@ struct anpd_kv {
     void* slab;
     size_t slab_bytes;
     bool staged;
+    int candidates;                   // 1, or 2: every step of the decoding loop verifies a second candidate too
     // one instantiated CUDA graph per distinct step shape (draft length, mode, attention grid)
     struct StepGraph { cudaGraphExec_t exec; int launches; };
     std::map<uint64_t, StepGraph> graphs;
@@ -390,7 +400,7 @@ struct anpd_kv {
 // max_pos: an upper bound of the largest position any row holds (sizes the attention grid).
 // head: also run the LM head and the per-block argmax (false for all but the last prefill pass).
 // head_row: in a prompt pass, the row whose next token is wanted (the LM head runs for its group of 8 rows only).
-anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits, int head_row = 0);
+anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, bool head, bool want_logits, int head_row = 0, bool two_candidates = false);
 
 // step_kernel.cu: the whole forward of a decode step as ONE persistent kernel (one CTA per SM).  True if this model / cache
 // pair can take that path (head dimension 128, one query head per kv head, dimensions that are multiples of 128).
@@ -400,15 +410,16 @@ anpd_status step_kernel_enqueue(anpd_model* m, anpd_kv* kv, int max_pos, bool wa
 void step_kernel_trace_dump(anpd_kv* kv);
 
 enum AcceptMode { ACCEPT_COMMIT = 0, ACCEPT_PEEK = 1, ACCEPT_PREFILL = 2 };
-anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv);
+anpd_status plan_decode_enqueue(anpd_model* m, anpd_kv* kv, bool two_candidates = false);
 anpd_status plan_prefill_enqueue(anpd_model* m, anpd_kv* kv, int seq, int start, int prompt_len, int rows);
 // mode COMMIT/PEEK: one block per sequence over its 8 rows.  PREFILL: `last_row` of sequence
 // `seq` gives the first generated token, kv_len becomes prompt_len.  d_ctxs may be null; otherwise
 // accepted tokens and the next token are appended to the sequences' token buffers.
-anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len);
+anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev* d_ctxs, int seq, int last_row, int prompt_len, bool two_candidates = false);
 
 // attn_tc.cu: per-page attention partials for head dimension 128 (same outputs as the mma.sync kernel in forward.cu)
-anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos);
+// tree: the rows carry cache slots and hidden slot ranges of their own (two-candidate steps)
+anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool tree = false);
 // attention of a prompt pass (one query head per kv head), written straight to the O projection's input
 anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows);
 

@@ -122,13 +122,13 @@ __global__ void ngram_bulk_kernel(NgramDev c, int from, int to) {
 // One block per sequence: fold the tokens committed since the last step (both passes), then
 // draft K tokens by chained back-off queries.  Warp w of the first n_max-n_min+1 warps serves
 // level n_max - w, so the levels of one query are probed side by side and the longest wins.
-__global__ void __launch_bounds__(STEP_THREADS) ngram_step_kernel(const NgramDev* ctxs, SeqState* seqs, int K) {
+__global__ void __launch_bounds__(STEP_THREADS) ngram_step_kernel(const NgramDev* ctxs, SeqState* seqs, int K, int K2) {
     pdl_trigger();
     pdl_wait();
     __shared__ NgramDev c;
     __shared__ int tail[ANPD_N_MAX - 1 + ANPD_K_MAX + 1];
-    __shared__ int res[ANPD_N_MAX];
-    __shared__ int s_avail, s_stop;
+    __shared__ int res[ANPD_N_MAX], res0[ANPD_N_MAX];
+    __shared__ int s_avail, s_stop, s_keep;
     if (threadIdx.x == 0) c = ctxs[blockIdx.x];
     __syncthreads();
     SeqState& sq = seqs[blockIdx.x];
@@ -149,6 +149,7 @@ __global__ void __launch_bounds__(STEP_THREADS) ngram_step_kernel(const NgramDev
         const int keep = min(T, c.n_max - 1);
         for (int i = 0; i < keep; ++i) tail[i] = c.tokens[T - keep + i];
         s_avail = keep;
+        s_keep = keep;
         s_stop = (T <= 0 || sq.active == 0) ? 1 : 0;
     }
     __syncthreads();
@@ -170,6 +171,7 @@ __global__ void __launch_bounds__(STEP_THREADS) ngram_step_kernel(const NgramDev
         if (threadIdx.x == 0) {
             int ans = -1;
             for (int w = 0; w < levels && ans < 0; ++w) ans = res[w];   // longest level first
+            if (i == 0) for (int w = 0; w < levels; ++w) res0[w] = res[w];
             if (ans < 0) s_stop = 1;
             else { tail[avail] = ans; s_avail = avail + 1; sq.draft[i] = ans; }
         }
@@ -180,6 +182,45 @@ __global__ void __launch_bounds__(STEP_THREADS) ngram_step_kernel(const NgramDev
         sq.draft_len = drafted;
         sq.last_tok = (T > 0) ? c.tokens[T - 1] : 0;
     }
+    // The second candidate: its first token is the answer of the longest level that disagrees with the first candidate's
+    // first token; it then continues like the first one, by back-off queries on its own temporary context.
+    int drafted2 = 0;
+    if (K2 > 0 && drafted > 0) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int alt = -1;
+            for (int w = 0; w < levels && alt < 0; ++w)
+                if (res0[w] >= 0 && res0[w] != sq.draft[0]) alt = res0[w];
+            s_stop = alt < 0 ? 1 : 0;
+            if (alt >= 0) { tail[s_keep] = alt; s_avail = s_keep + 1; sq.draft2[0] = alt; }
+        }
+        __syncthreads();
+        if (!s_stop) drafted2 = 1;
+        for (int i = 1; i < K2; ++i) {
+            if (s_stop) break;
+            const int avail = s_avail;
+            if (warp < levels) {
+                const int n = c.n_max - warp, klen = n - 1;
+                int ans = -1;
+                if (avail >= klen) {
+                    const int s = warp_probe<PrefSlot, false>(c.pref[n], c.cap, c.tokens, tail + avail - klen, klen, n, 0);
+                    if (s >= 0) ans = (int)(*((volatile unsigned long long*)&c.pref[n][s].best) & 0xFFFFFFull);
+                    if (s == -2 && (threadIdx.x & 31) == 0) atomicExch(&c.state[2], NG_ERR_FULL);
+                }
+                if ((threadIdx.x & 31) == 0) res[warp] = ans;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int ans = -1;
+                for (int w = 0; w < levels && ans < 0; ++w) ans = res[w];
+                if (ans < 0) s_stop = 1;
+                else { tail[avail] = ans; s_avail = avail + 1; sq.draft2[i] = ans; }
+            }
+            __syncthreads();
+            if (!s_stop) ++drafted2;
+        }
+    }
+    if (threadIdx.x == 0) sq.draft2_len = drafted2;
 }
 
 int next_pow2(int v) { int p = 64; while (p < v) p <<= 1; return p; }
@@ -200,8 +241,8 @@ anpd_status ngram_enqueue_bulk(anpd_ngram* ctx, int from, int to, Profiler* prof
 }
 
 anpd_status ngram_enqueue_step(const NgramDev* d_ctxs, SeqState* d_seq, int batch, int K,
-                               cudaStream_t st, Profiler* prof) {
-    LAUNCH(prof, st, KC_NGRAM, 0, (launch_k(ngram_step_kernel, batch, STEP_THREADS, 0, st, d_ctxs, d_seq, K)));
+                               cudaStream_t st, Profiler* prof, int K2) {
+    LAUNCH(prof, st, KC_NGRAM, 0, (launch_k(ngram_step_kernel, batch, STEP_THREADS, 0, st, d_ctxs, d_seq, K, K2)));
     CUDA_TRY(cudaGetLastError());
     return ANPD_OK;
 }

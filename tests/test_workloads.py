@@ -104,3 +104,36 @@ def test_orbit_model_continues_its_orbit_under_the_oracle_decoder():
     assert (st.steps, st.drafted, st.accepted, st.hist_accepted, st.drafts, st.accepted_lens) == \
            (st2.steps, st2.drafted, st2.accepted, st2.hist_accepted, st2.drafts, st2.accepted_lens)
     assert 0.3 < st.hit_ratio < 0.8
+
+
+def test_forked_orbit_prompt_makes_the_second_candidate_win():
+    """orbit_fork_prompt: the stretch appears three times with the promised edits (a wrong successor once, an inserted
+    token twice) and ends on the stretch's first token; under the oracle the one-candidate loop drafts the wrong token
+    at every fork while the two-candidate loop's alternative is accepted there, so it takes fewer steps; the scripted
+    stand-in and the real decoder on the orbit weights take the same steps."""
+    from oracle.anpd import anpd_generate, anpd_generate_two_candidates
+    from oracle.decoder import Decoder
+    from workloads import ScriptedOrbitModel, make_orbit_weights, orbit_continuation, orbit_fork_prompt, orbit_permutation
+    pi = orbit_permutation(211, 9)
+    p = orbit_fork_prompt(pi, 150, 4, every=7).tolist()
+    assert len(p) == 150 and p == orbit_fork_prompt(pi, 150, 4, every=7).tolist()
+    # the last token opens the stretch; the stretch's second token follows it somewhere in the prompt
+    first = p[-1]
+    assert sum(1 for i in range(149) if p[i] == first and p[i + 1] == int(pi[first])) == 3
+    # transitions that follow the orbit dominate; the edits are a minority
+    on_orbit = sum(1 for i in range(149) if int(pi[p[i]]) == p[i + 1])
+    assert 0.6 * 149 < on_orbit < 149
+    mdl = ScriptedOrbitModel(pi, 256)
+    want = orbit_continuation(pi, p[-1], 40).tolist()
+    for policy in (0, 1):
+        o1, s1, _ = anpd_generate(mdl, p, 40, 4, n_max=4, policy=policy)
+        o2, s2, _ = anpd_generate_two_candidates(mdl, p, 40, 4, n_max=4, policy=policy)
+        assert o1 == want and o2 == want
+        assert s2.alt_wins >= 3 and s2.steps < s1.steps
+    wl = WORKLOADS["C1-A50"]
+    w, pi2 = make_orbit_weights(wl.shape, wl.weight_seed, wl.orbit_S, bf16=wl.weights_bf16)
+    q = orbit_fork_prompt(pi2, wl.prompt_len, wl.prompt_seed).tolist()
+    a, sa, _ = anpd_generate_two_candidates(Decoder(wl.shape, w, torch.float64), q, 32, 4, n_max=wl.n_max)
+    b, sb, _ = anpd_generate_two_candidates(ScriptedOrbitModel(pi2, wl.shape.vocab), q, 32, 4, n_max=wl.n_max)
+    assert a == b == orbit_continuation(pi2, q[-1], 32).tolist()
+    assert (sa.steps, sa.drafts, sa.accepted_lens, sa.alt_wins) == (sb.steps, sb.drafts, sb.accepted_lens, sb.alt_wins) and sa.alt_wins > 0

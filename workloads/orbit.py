@@ -70,6 +70,39 @@ def orbit_prompt(pi: np.ndarray, length: int, corrupt: float, seed: int, replay_
     return np.asarray(out, dtype=np.int32)
 
 
+def orbit_fork_prompt(pi: np.ndarray, length: int, seed: int, every: int = 9) -> np.ndarray:
+    """int32[length]: a stretch of the orbit shown three times, closed by the stretch's first token, built so that at
+    every `every`-th token d of the stretch (predecessor c, successor e) a decoding step STARTS at d with n-gram
+    tables whose long contexts are misleading and whose one-token context is right:
+      - the first showing replaces e by a random token x: the only time d stood behind c it was followed by x;
+      - the other two showings insert a token z between c and d: c is followed by z twice (so the draft made at c is
+        wrong and the next step starts at d), and d, now behind z, is followed by e twice.
+    A module that verifies one candidate drafts x after d; one that also verifies the answer of a shorter level drafts e
+    as well.  Leading tokens, if any, are random filler."""
+    S = len(pi)
+    L = 8
+    while 3 * (L + 1) + 2 * len(range(4, L + 1 - 2, every)) + 1 <= length:
+        L += 1
+    forks = list(range(4, L - 2, every))
+    t = randint_at(seed, _S_NOISE, 0, 0, S - 1)
+    stretch = []
+    for _ in range(L):
+        stretch.append(t)
+        t = int(pi[t])
+    def other(k, avoid):
+        r = randint_at(seed, _S_NOISE, 1 + k, 0, S - 1)
+        return r if r != avoid else (r + 1) % S
+    body = []
+    for rep in range(3):
+        for i, tok in enumerate(stretch):
+            if rep > 0 and i in forks:
+                body.append(other(2 * i, stretch[i]))                   # z: the same in both showings
+            body.append(other(2 * i + 1, tok) if (rep == 0 and i - 1 in forks) else tok)
+    body.append(stretch[0])
+    fill = [randint_at(seed, _S_NOISE, 1 + 2 * L + k, 0, S - 1) for k in range(length - len(body))]
+    return np.asarray(fill + body, dtype=np.int32)
+
+
 def orbit_continuation(pi: np.ndarray, last_tok: int, n: int) -> np.ndarray:
     """The model's greedy output after a prompt ending in last_tok: pi(last), pi^2(last), ..."""
     out, t = [], int(last_tok)
