@@ -206,40 +206,69 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         if (t == 0) { load_page(&map_v, &bar_v[slot], cur); ++v_issued; }
         uint4 qr[QCH];
         if (more) fetch_q(nxt, qr);
-        float s[Q];
-        {
-            float v[N];
-#pragma unroll
-            for (int c0 = 0; c0 < N; c0 += 16) tc_ld16(lane_base + (uint32_t)c0, v + c0);
-#pragma unroll
-            for (int q = 0; q < Q; ++q) s[q] = v[q] + v[Q + q];
-        }
-        // mask by position (this thread's key is c * 128 + t), maximum over the page's keys per query vector
+        // Scores of this thread's key (c * 128 + t) for QC query vectors at a time, masked by position.  With up to 16
+        // query vectors (1 or 2 query heads per kv head) they stay in registers across the barrier; with more they are
+        // read from tensor memory a second time instead (the second product overwrites them only after the barrier
+        // behind the P operand), which keeps the kernel out of local memory.
+        constexpr int QC = Q < 16 ? Q : 16;
         const int key = cur.c * KV_PAGE + t;
+        auto scores = [&](int q0, float* s) {
+            float v[2 * QC];
+            if constexpr (Q <= 8) {
+                tc_ld16(lane_base, v);                                           // hi terms 0..7, lo terms 8..15
+            } else {
+                tc_ld16(lane_base + (uint32_t)q0, v);
+                tc_ld16(lane_base + (uint32_t)(Q + q0), v + QC);
+            }
 #pragma unroll
-        for (int q = 0; q < Q; ++q) {
-            if (key > cur.pos_lo + (q & 7)) s[q] = -CUDART_INF_F;
-            if (row_slot && key >= row_hole_lo[cur.r0 + (q & 7)] && key < row_hole_hi[cur.r0 + (q & 7)]) s[q] = -CUDART_INF_F;
-            float mx = s[q];
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            if (lane == 0) red_max[slot][warp][q] = mx;
+            for (int q = 0; q < QC; ++q) {
+                s[q] = v[q] + v[QC + q];
+                if (key > cur.pos_lo + (q & 7)) s[q] = -CUDART_INF_F;           // q0 is a multiple of 8: (q0 + q) & 7 == q & 7
+                if (row_slot && key >= row_hole_lo[cur.r0 + (q & 7)] && key < row_hole_hi[cur.r0 + (q & 7)]) s[q] = -CUDART_INF_F;
+            }
+        };
+        float s_keep[QC];
+        // maximum over the page's keys per query vector
+#pragma unroll
+        for (int q0 = 0; q0 < Q; q0 += QC) {
+            float s[QC];
+            scores(q0, s);
+#pragma unroll
+            for (int q = 0; q < QC; ++q) {
+                float mx = s[q];
+                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                if (lane == 0) red_max[slot][warp][q0 + q] = mx;
+                if (Q <= 16) s_keep[q] = s[q];
+            }
         }
         tc_fence_before();
         slot_bar(slot);
+        if constexpr (Q > 16) tc_fence_after();
         // weights (base-2 domain: the queries carry log2(e) / sqrt(hd)), their sum, and the P operand
-        float m[Q];
 #pragma unroll
-        for (int q = 0; q < Q; ++q) {
-            m[q] = fmaxf(fmaxf(red_max[slot][0][q], red_max[slot][1][q]), fmaxf(red_max[slot][2][q], red_max[slot][3][q]));
-            const float p = (m[q] == -CUDART_INF_F) ? 0.0f : exp2f(s[q] - m[q]);
-            const bf16 h = __float2bfloat16_rn(p);
-            const bf16 l = __float2bfloat16_rn(p - __bfloat162float(h));
-            *(bf16*)(Ps + b_operand_offset<N>(q, t)) = h;
-            *(bf16*)(Ps + b_operand_offset<N>(Q + q, t)) = l;
-            float sum = p;
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) red_sum[slot][par][warp][q] = sum;
+        for (int q0 = 0; q0 < Q; q0 += QC) {
+            float s[QC];
+            if constexpr (Q <= 16) {
+#pragma unroll
+                for (int q = 0; q < QC; ++q) s[q] = s_keep[q];
+            } else {
+                scores(q0, s);
+            }
+#pragma unroll
+            for (int q = 0; q < QC; ++q) {
+                const int qq = q0 + q;
+                const float m = fmaxf(fmaxf(red_max[slot][0][qq], red_max[slot][1][qq]), fmaxf(red_max[slot][2][qq], red_max[slot][3][qq]));
+                const float p = (m == -CUDART_INF_F) ? 0.0f : exp2f(s[q] - m);
+                const bf16 h = __float2bfloat16_rn(p);
+                const bf16 l = __float2bfloat16_rn(p - __bfloat162float(h));
+                *(bf16*)(Ps + b_operand_offset<N>(qq, t)) = h;
+                *(bf16*)(Ps + b_operand_offset<N>(Q + qq, t)) = l;
+                float sum = p;
+                for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+                if (lane == 0) red_sum[slot][par][warp][qq] = sum;
+            }
         }
+        if constexpr (Q > 16) tc_fence_before();          // the scores were read again: order those reads before the second product
         if (more) stage_q(qr);
         fence_async_smem();
         slot_bar(slot);
@@ -258,23 +287,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
         }
         if (t < Q) {
             const size_t out = ((size_t)(cur.r0 + (t & 7)) * Hq + (cur.kvh * G + (t >> 3))) * pages_per_seq + cur.c;
-            float mt = m[0];
-#pragma unroll
-            for (int q = 1; q < Q; ++q) mt = (q == t) ? m[q] : mt;
-            pm[out] = mt;
+            pm[out] = fmaxf(fmaxf(red_max[slot][0][t], red_max[slot][1][t]), fmaxf(red_max[slot][2][t], red_max[slot][3][t]));
             pl[out] = (red_sum[slot][par][0][t] + red_sum[slot][par][1][t]) + (red_sum[slot][par][2][t] + red_sum[slot][par][3][t]);
         }
         mbar_wait(&bar_o[slot], par, abortp);
         tc_fence_after();
         if (more && t == 0) { load_page(&map_k, &bar_k[slot], nxt); ++k_issued; }        // the second product is done with the page buffer
-        {
-            float v[N];
 #pragma unroll
-            for (int c0 = 0; c0 < N; c0 += 16) tc_ld16(lane_base + (uint32_t)c0, v + c0);
+        for (int q0 = 0; q0 < Q; q0 += QC) {
+            float v[2 * QC];
+            if constexpr (Q <= 8) {
+                tc_ld16(lane_base, v);
+            } else {
+                tc_ld16(lane_base + (uint32_t)q0, v);
+                tc_ld16(lane_base + (uint32_t)(Q + q0), v + QC);
+            }
 #pragma unroll
-            for (int q = 0; q < Q; ++q) {
-                const size_t out = ((size_t)(cur.r0 + (q & 7)) * Hq + (cur.kvh * G + (q >> 3))) * pages_per_seq + cur.c;
-                po[out * HD + t] = v[q] + v[Q + q];
+            for (int q = 0; q < QC; ++q) {
+                const int qq = q0 + q;
+                const size_t out = ((size_t)(cur.r0 + (qq & 7)) * Hq + (cur.kvh * G + (qq >> 3))) * pages_per_seq + cur.c;
+                po[out * HD + t] = v[q] + v[QC + q];
             }
         }
         tc_fence_before();
