@@ -158,7 +158,7 @@ static anpd_status model_make_plans(anpd_model* m) {
         max_tiles = std::max(max_tiles, m->plan[k].m_tiles);
         m->max_segs = std::max(m->max_segs, m->plan[k].max_segs);
     }
-    ints += 4 * (size_t)max_tiles;
+    ints += 4 * (size_t)max_tiles + (size_t)GK_COUNT * max_tiles;
     std::vector<int> host(ints);
     CUDA_TRY(cudaMalloc((void**)&m->d_plan_tables, ints * sizeof(int)));
     size_t off = 0;
@@ -175,6 +175,10 @@ static anpd_status model_make_plans(anpd_model* m) {
     for (int k = 2; k <= 3; ++k) {
         m->d_const_segs[k] = m->d_plan_tables + off + (size_t)(k - 1) * max_tiles;
         for (int i = 0; i < max_tiles; ++i) host[off + (size_t)(k - 1) * max_tiles + i] = k;
+    }
+    for (int k = 0; k < GK_COUNT; ++k) {
+        m->d_tail_segs[k] = m->d_plan_tables + off + (size_t)(3 + k) * max_tiles;
+        m->tail_cfg[k] = -1;
     }
     CUDA_TRY(cudaMemcpy(m->d_plan_tables, host.data(), ints * sizeof(int), cudaMemcpyHostToDevice));
     return ANPD_OK;

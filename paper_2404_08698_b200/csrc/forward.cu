@@ -922,6 +922,14 @@ __global__ void __launch_bounds__(256) gemm_rows8_kernel(const bf16* __restrict_
     }
 }
 
+// segment counts of a prompt-pass projection whose last tiles alone are cut along K
+__global__ void fill_tail_segs_kernel(int* segs, int m_tiles, int first_cut, int parts) {
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < m_tiles) segs[i] = i >= first_cut ? parts : 1;
+}
+
 // rows [from, from + 8) of the normalised activations -> rows [0, 8)
 __global__ void move_rows_kernel(bf16* __restrict__ h_hi, bf16* __restrict__ h_lo, int from, int d) {
     pdl_trigger();
@@ -950,10 +958,21 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
         return gemm_plain_enqueue(plan, W, a_hi, a_lo, rows, ws.part, ws.n_max_out, m->stream, &m->prof);
     }
     if (mode == 1) {                                   // a prompt pass: complete sums, one per output
-        const int n_tiles = ((plan.m_tiles + 1) / 2) * ((rows + 255) / 256);
-        const int ksplit = gemm_pf_ksplit(n_tiles, plan.k_blocks, m->num_sms);
-        *seg_count_out = m->d_const_segs[ksplit];
-        return gemm_pf_enqueue(plan, W, maps[0], maps[1], rows, ws.part, ws.n_max_out, (size_t)ws.r_max * ws.n_max_out, ksplit, m->num_sms,
+        const int n_ft = (plan.m_tiles + 1) / 2, n_tt = (rows + 255) / 256;
+        const PfSchedule sched = gemm_pf_schedule(n_ft, n_tt, plan.k_blocks, m->num_sms);
+        if (sched.tail_split > 1) {                    // feature tiles from `first` on come in tail_split parts, the others in one
+            const int first = 2 * (sched.tail_from / n_tt), cfg = first * 4 + sched.tail_split;
+            if (m->tail_cfg[kind] != cfg) {
+                LAUNCH(&m->prof, m->stream, KC_OTHER, 0,
+                       (launch_k(fill_tail_segs_kernel, (plan.m_tiles + 127) / 128, 128, 0, m->stream, m->d_tail_segs[kind], plan.m_tiles, first,
+                                 sched.tail_split)));
+                m->tail_cfg[kind] = cfg;
+            }
+            *seg_count_out = m->d_tail_segs[kind];
+        } else {
+            *seg_count_out = m->d_const_segs[sched.ksplit];
+        }
+        return gemm_pf_enqueue(plan, W, maps[0], maps[1], rows, ws.part, ws.n_max_out, (size_t)ws.r_max * ws.n_max_out, sched, m->num_sms,
                                ws.gemm_err, m->stream, &m->prof);
     }
     ANPD_TRY(gemm_tc_enqueue(plan, W, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)kv->batch * ANPD_ROWS * ws.n_max_out,

@@ -9,11 +9,14 @@
 // against 256 rows.  Tiles that share a weight pair run on neighbouring CTAs at the same time, so a weight block crosses HBM
 // once per prompt pass and is served from L2 otherwise.  A projection with fewer tiles than would keep every SM busy is also cut
 // along K into `ksplit` equal parts (the same cut for every tile): part s leaves its sums in partial-sum slab s and the
-// consumers add the slabs in order, as they add the decode GEMM's segments.
+// consumers add the slabs in order, as they add the decode GEMM's segments.  A projection whose tiles fill some rounds of
+// CTAs and a fraction of one more has the tiles of that last round alone cut into 2 or 3 parts, so that the round takes a
+// half or a third of a tile's time on all SMs instead of a whole tile's time on some.
 #include "internal.h"
 #include "tc_ptx.cuh"
 
 #include <algorithm>
+#include <vector>
 
 typedef __nv_bfloat16 bf16;
 
@@ -32,10 +35,18 @@ struct PfArgs {
     float* out; int ld;
     int N, rows;
     int m_tiles, k_blocks, n_ft, n_tt, ksplit;
+    int tail_from, tail_split;         // output tiles from tail_from on are cut into tail_split parts instead of ksplit
     size_t seg_stride;                 // elements between the partial-sum slabs of two K parts
     long long total; int G;
     int* err;
 };
+
+// work item -> (output tile, K part, parts of that tile); K part fastest
+__device__ __forceinline__ void pf_item(const PfArgs& g, int item, int& ot, int& ks, int& parts) {
+    const int uniform = g.tail_from * g.ksplit;
+    if (item < uniform) { ot = item / g.ksplit; ks = item - ot * g.ksplit; parts = g.ksplit; }
+    else { const int j = item - uniform; ot = g.tail_from + j / g.tail_split; ks = j % g.tail_split; parts = g.tail_split; }
+}
 
 __global__ void __launch_bounds__(PF_THREADS, 1)
 gemm_pf_kernel(const bf16* __restrict__ w_blocks, const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
@@ -48,7 +59,7 @@ gemm_pf_kernel(const bf16* __restrict__ w_blocks, const __grid_constant__ CUtens
     pdl_trigger();
     unsigned char* smem = pf_smem_raw + ((1024u - (smem_u32(pf_smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = g.n_ft * g.n_tt * g.ksplit;     // work items: (feature pair, row tile, K part), K part fastest
+    const int n_tiles = g.tail_from * g.ksplit + (g.n_ft * g.n_tt - g.tail_from) * g.tail_split;     // work items
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -77,12 +88,13 @@ gemm_pf_kernel(const bf16* __restrict__ w_blocks, const __grid_constant__ CUtens
             long long issued = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int ks = tile % g.ksplit, ot = tile / g.ksplit;
+                int ot, ks, parts;
+                pf_item(g, tile, ot, ks, parts);
                 const int ft = ot / g.n_tt, tt = ot - ft * g.n_tt;
                 const int t0 = 2 * ft, t1 = min(2 * ft + 1, g.m_tiles - 1);      // an odd tile count: the last pair repeats its tile
                 const int row0 = tt * PF_TILE_TOK;
-                const int kb_end = (int)((long long)(ks + 1) * g.k_blocks / g.ksplit);
-                for (int kb = (int)((long long)ks * g.k_blocks / g.ksplit); kb < kb_end; ++kb) {
+                const int kb_end = (int)((long long)(ks + 1) * g.k_blocks / parts);
+                for (int kb = (int)((long long)ks * g.k_blocks / parts); kb < kb_end; ++kb) {
                     ok = mbar_wait(&bar_empty[stage], phase ^ 1u, abortp);
                     if (!ok) break;
                     unsigned char* st = smem + (size_t)stage * PF_STAGE;
@@ -120,8 +132,9 @@ gemm_pf_kernel(const bf16* __restrict__ w_blocks, const __grid_constant__ CUtens
                 ok = mbar_wait(&bar_acc_empty, (uint32_t)((done_tiles & 1) ^ 1), abortp);      // the epilogue has read the previous tile
                 if (!ok) break;
                 tc_fence_after();
-                const int ks = tile % g.ksplit;
-                const int kb_begin = (int)((long long)ks * g.k_blocks / g.ksplit), kb_end = (int)((long long)(ks + 1) * g.k_blocks / g.ksplit);
+                int ot, ks, parts;
+                pf_item(g, tile, ot, ks, parts);
+                const int kb_begin = (int)((long long)ks * g.k_blocks / parts), kb_end = (int)((long long)(ks + 1) * g.k_blocks / parts);
                 for (int kb = kb_begin; kb < kb_end; ++kb) {
                     ok = mbar_wait(&bar_full[stage], phase, abortp);
                     if (!ok) break;
@@ -152,7 +165,8 @@ gemm_pf_kernel(const bf16* __restrict__ w_blocks, const __grid_constant__ CUtens
         int done_tiles = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++done_tiles) {
-            const int ks = tile % g.ksplit, ot = tile / g.ksplit;
+            int ot, ks, parts;
+            pf_item(g, tile, ot, ks, parts);
             const int ft = ot / g.n_tt, tt = ot - ft * g.n_tt;
             ok = mbar_wait(&bar_acc_full, (uint32_t)(done_tiles & 1), abortp);
             if (!ok) break;
@@ -194,21 +208,44 @@ gemm_pf_kernel(const bf16* __restrict__ w_blocks, const __grid_constant__ CUtens
 
 }  // namespace
 
-// Cuts of K for a projection with `tiles` output tiles of which each takes `k_blocks` steps: the cut (1, 2 or 3 parts) with the
-// fewest steps on the busiest SM.
-int gemm_pf_ksplit(int tiles, int k_blocks, int num_sms) {
-    int best = 1;
-    long long best_cost = 0;
-    for (int s = 1; s <= 3; ++s) {
-        const long long rounds = ((long long)tiles * s + num_sms - 1) / num_sms;
-        const long long cost = rounds * ((k_blocks + s - 1) / s) + rounds * 6;      // + the epilogue of every round, about six steps' worth
-        if (s == 1 || cost < best_cost) { best = s; best_cost = cost; }
+// Steps on the busiest CTA when the work items go to the CTAs round robin (a tile's epilogue counts as about six steps).
+static long long pf_cost(int n_ot, int k_blocks, int num_sms, const PfSchedule& s) {
+    const int uniform = s.tail_from * s.ksplit;
+    const int n_items = uniform + (n_ot - s.tail_from) * s.tail_split;
+    const int grid = std::min(num_sms, n_items);
+    std::vector<long long> load((size_t)grid, 0);
+    for (int it = 0; it < n_items; ++it) {
+        const int parts = it < uniform ? s.ksplit : s.tail_split;
+        load[(size_t)(it % grid)] += (k_blocks + parts - 1) / parts + 6;
+    }
+    return *std::max_element(load.begin(), load.end());
+}
+
+// The cut along K with the fewest steps on the busiest SM: every tile in 1, 2 or 3 parts, or the tiles of the last, partly
+// filled round alone in 2 or 3 parts.
+PfSchedule gemm_pf_schedule(int n_ft, int n_tt, int k_blocks, int num_sms) {
+    const int n_ot = n_ft * n_tt;
+    PfSchedule best{1, n_ot, 1};
+    long long best_cost = pf_cost(n_ot, k_blocks, num_sms, best);
+    for (int s = 2; s <= 3; ++s) {
+        const PfSchedule c{s, n_ot, 1};
+        const long long cost = pf_cost(n_ot, k_blocks, num_sms, c);
+        if (cost < best_cost) { best = c; best_cost = cost; }
+    }
+    const int full = n_ot / num_sms;
+    if (full >= 1 && n_ot % num_sms != 0) {
+        const int from = (full * num_sms / n_tt) * n_tt;            // whole feature pairs stay uncut
+        for (int s = 2; s <= 3 && from > 0; ++s) {
+            const PfSchedule c{1, from, s};
+            const long long cost = pf_cost(n_ot, k_blocks, num_sms, c);
+            if (cost < best_cost) { best = c; best_cost = cost; }
+        }
     }
     return best;
 }
 
 anpd_status gemm_pf_enqueue(const GemmPlan& plan, const bf16* w_blocks, const CUtensorMap& map_hi, const CUtensorMap& map_lo, int rows,
-                            float* out, int ld, size_t seg_stride, int ksplit, int num_sms, int* err, cudaStream_t st, Profiler* prof) {
+                            float* out, int ld, size_t seg_stride, PfSchedule sched, int num_sms, int* err, cudaStream_t st, Profiler* prof) {
     constexpr int smem = PF_STAGES * PF_STAGE + 1024;
     static bool attr_set[64] = {false};
     if (first_call_on_device(attr_set)) {
@@ -221,9 +258,9 @@ anpd_status gemm_pf_enqueue(const GemmPlan& plan, const bf16* w_blocks, const CU
     g.n_tt = (rows + PF_TILE_TOK - 1) / PF_TILE_TOK;
     g.total = (long long)plan.m_tiles * plan.k_blocks;
     g.G = plan.grid;
-    g.ksplit = ksplit; g.seg_stride = seg_stride;
+    g.ksplit = sched.ksplit; g.tail_from = sched.tail_from; g.tail_split = sched.tail_split; g.seg_stride = seg_stride;
     g.err = err;
-    const int grid = std::min(num_sms, g.n_ft * g.n_tt * ksplit);
+    const int grid = std::min(num_sms, sched.tail_from * sched.ksplit + (g.n_ft * g.n_tt - sched.tail_from) * sched.tail_split);
     LAUNCH(prof, st, KC_GEMM, 2.0 * (double)plan.N * (double)plan.K,
            (launch_k(gemm_pf_kernel, grid, PF_THREADS, (size_t)smem, st, w_blocks, map_hi, map_lo, g)));
     CUDA_TRY(cudaGetLastError());

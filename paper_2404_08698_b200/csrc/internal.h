@@ -269,6 +269,8 @@ struct anpd_model {
     int* d_plan_tables;               // device copies of the plans' tables
     int* d_ones;                      // [tiles] all 1: segment counts of the plain GEMM
     int* d_const_segs[4];             // [tiles] all k (k = 1..3): segment counts of a prompt-pass GEMM cut into k parts along K
+    int* d_tail_segs[GK_COUNT];       // [tiles] segment counts of a prompt-pass GEMM whose last tiles alone are cut (PfSchedule)
+    int tail_cfg[GK_COUNT];           // what d_tail_segs[kind] holds: first cut feature tile * 4 + parts, -1 = nothing yet
     int max_segs;
     bool plain_gemm;                  // debugging aid: route GEMMs through the plain kernel
     // second copy of the projections in row-range storage, used by single-sequence steps (proj_rr.cu)
@@ -448,10 +450,14 @@ anpd_status gemm_tc_enqueue(const GemmPlan& plan, const __nv_bfloat16* w_blocks,
                             int rows, int NB, float* part, size_t seg_stride, int ld_part, int* err, cudaStream_t st,
                             Profiler* prof);
 // gemm_pf.cu: the projection of a prompt pass (many rows, bound by the tensor cores): out[row][n], complete sums
-// out[part][row][n]: `ksplit` partial sums per output, seg_stride elements apart (gemm_pf_ksplit picks the cut)
-int gemm_pf_ksplit(int tiles, int k_blocks, int num_sms);
+// out[part][row][n]: partial sums per output, seg_stride elements apart.  How the output tiles (feature pair x row tile, row
+// tile fastest) are cut along K: tiles [0, tail_from) into `ksplit` equal parts each, tiles [tail_from, end) - those that would
+// form a last, partly filled round of CTAs - into `tail_split` parts (tail_from == tile count: no such tail; a multiple of the
+// row tile count, so that a feature tile has one part count for all its rows).
+struct PfSchedule { int ksplit, tail_from, tail_split; };
+PfSchedule gemm_pf_schedule(int n_ft, int n_tt, int k_blocks, int num_sms);
 anpd_status gemm_pf_enqueue(const GemmPlan& plan, const __nv_bfloat16* w_blocks, const CUtensorMap& map_hi, const CUtensorMap& map_lo, int rows,
-                            float* out, int ld, size_t seg_stride, int ksplit, int num_sms, int* err, cudaStream_t st, Profiler* prof);
+                            float* out, int ld, size_t seg_stride, PfSchedule sched, int num_sms, int* err, cudaStream_t st, Profiler* prof);
 // forward.cu: the plain (one warp per output feature) GEMM, kept as a cross-check
 anpd_status gemm_plain_enqueue(const GemmPlan& p, const __nv_bfloat16* W, const __nv_bfloat16* a_hi, const __nv_bfloat16* a_lo, int rows,
                                float* part, int ld_part, cudaStream_t st, Profiler* prof);
