@@ -271,13 +271,23 @@ __global__ void __launch_bounds__(256) qkv_rope_append_tile_kernel(const float* 
     const int ns = seg_count[(head * HD) >> 7];          // a head never straddles a 128-column tile
     // 16-byte loads, eight of them in flight per thread
     constexpr int Q4 = HD / 4;
-#pragma unroll 8
-    for (int idx = threadIdx.x; idx < nr * Q4; idx += 256) {
-        const int r = idx / Q4, dim = (idx % Q4) * 4;
-        const float* pr = part + (size_t)(r0 + r) * ld_part + (size_t)head * HD + dim;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < ns; ++s) { const float4 v = *(const float4*)(pr + s * split_stride); a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
-        tile[r][dim] = a.x; tile[r][dim + 1] = a.y; tile[r][dim + 2] = a.z; tile[r][dim + 3] = a.w;
+    for (int base = 0; base < nr * Q4; base += 8 * 256) {
+        float4 a[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {                     // the first partial sums (there is always one): eight independent loads
+            const int idx = base + u * 256 + threadIdx.x;
+            a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (idx < nr * Q4) a[u] = *(const float4*)(part + (size_t)(r0 + idx / Q4) * ld_part + (size_t)head * HD + (idx % Q4) * 4);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + threadIdx.x;
+            if (idx >= nr * Q4) continue;
+            const int r = idx / Q4, dim = (idx % Q4) * 4;
+            const float* pr = part + (size_t)(r0 + r) * ld_part + (size_t)head * HD + dim;
+            for (int s = 1; s < ns; ++s) { const float4 v = *(const float4*)(pr + s * split_stride); a[u].x += v.x; a[u].y += v.y; a[u].z += v.z; a[u].w += v.w; }
+            tile[r][dim] = a[u].x; tile[r][dim + 1] = a[u].y; tile[r][dim + 2] = a[u].z; tile[r][dim + 3] = a[u].w;
+        }
     }
     __syncthreads();
     if (head < Hq + Hkv) {
@@ -715,19 +725,39 @@ __global__ void swiglu_wide_kernel(const float* __restrict__ part, const int* __
                                    bf16* __restrict__ act_hi, bf16* __restrict__ act_lo) {
     pdl_trigger();
     pdl_wait();
-    const int row = blockIdx.y, j = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
-    if (j >= F) return;
+    // two chunks of four features per thread (a block's width apart); every output has at least one partial sum, so the
+    // first partial sums of gate and up of both chunks are requested together, before anything depends on them
+    const int row = blockIdx.y, j0 = 4 * (2 * blockIdx.x * blockDim.x + threadIdx.x);
     const float* pr = part + (size_t)row * ld_part;
-    float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), u4 = g4;
-    const int ng = seg_count[j >> 7], nu = seg_count[(F + j) >> 7];
-    for (int s = 0; s < ng; ++s) { const float4 p = *(const float4*)(pr + s * split_stride + j); g4.x += p.x; g4.y += p.y; g4.z += p.z; g4.w += p.w; }
-    for (int s = 0; s < nu; ++s) { const float4 p = *(const float4*)(pr + s * split_stride + F + j); u4.x += p.x; u4.y += p.y; u4.z += p.z; u4.w += p.w; }
-    const float gte[4] = {g4.x, g4.y, g4.z, g4.w}, up[4] = {u4.x, u4.y, u4.z, u4.w};
-    bf16 hi[4], lo[4];
+    float4 g4[2], u4[2];
+    int ng[2], nu[2];
+    bool live[2];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) split_bf16(gte[e] / (1.0f + expf(-gte[e])) * up[e], hi[e], lo[e]);
-    *(uint2*)(act_hi + (size_t)row * F + j) = *(const uint2*)hi;
-    *(uint2*)(act_lo + (size_t)row * F + j) = *(const uint2*)lo;
+    for (int c = 0; c < 2; ++c) {
+        const int j = j0 + c * 4 * blockDim.x;
+        live[c] = j < F;
+        g4[c] = u4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        ng[c] = nu[c] = 0;
+        if (live[c]) {
+            g4[c] = *(const float4*)(pr + j);
+            u4[c] = *(const float4*)(pr + F + j);
+            ng[c] = seg_count[j >> 7];
+            nu[c] = seg_count[(F + j) >> 7];
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        if (!live[c]) continue;
+        const int j = j0 + c * 4 * blockDim.x;
+        for (int s = 1; s < ng[c]; ++s) { const float4 p = *(const float4*)(pr + s * split_stride + j); g4[c].x += p.x; g4[c].y += p.y; g4[c].z += p.z; g4[c].w += p.w; }
+        for (int s = 1; s < nu[c]; ++s) { const float4 p = *(const float4*)(pr + s * split_stride + F + j); u4[c].x += p.x; u4[c].y += p.y; u4[c].z += p.z; u4[c].w += p.w; }
+        const float gte[4] = {g4[c].x, g4[c].y, g4[c].z, g4[c].w}, up[4] = {u4[c].x, u4[c].y, u4[c].z, u4[c].w};
+        bf16 hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) split_bf16(gte[e] / (1.0f + expf(-gte[e])) * up[e], hi[e], lo[e]);
+        *(uint2*)(act_hi + (size_t)row * F + j) = *(const uint2*)hi;
+        *(uint2*)(act_lo + (size_t)row * F + j) = *(const uint2*)lo;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1157,7 +1187,7 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
                                                        ws.h_hi, ws.h_lo)));
         ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs));
         if (many_rows) LAUNCH(pf, st, KC_OTHER, 0,
-               (launch_k(swiglu_wide_kernel, dim3((F / 4 + 255) / 256, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
+               (launch_k(swiglu_wide_kernel, dim3((F / 4 + 511) / 512, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
                          ws.act_lo)));
         else LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(swiglu_kernel, dim3((F + 255) / 256, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
