@@ -208,3 +208,65 @@ def test_two_candidate_host_stepped_loop_equals_device_loop(A, monkeypatch):
     s_host, _ = run_fork_workload(A, "C1-A50", f, 5)
     for k in ("steps", "drafted", "accepted", "alt_wins", "hist_accepted", "generated"):
         assert s_dev[k] == s_host[k]
+
+
+def test_two_candidate_batch_equals_independent_runs(A):
+    """Three sequences in one kv handle (shuffled pages), each with its own forked prompt: the batched two-candidate
+    loop gives every sequence the stream and statistics of its own single-sequence run and of the oracle."""
+    wl = WORKLOADS["C1-A50"]
+    w, pi = make_orbit_weights(wl.shape, wl.weight_seed, wl.orbit_S, bf16=wl.weights_bf16)
+    st = new_stream()
+    m = gpu_model(A, wl.shape, w, st)
+    B, M, K = 3, 48, 5
+    prompts = np.stack([orbit_fork_prompt(pi, wl.prompt_len, 300 + b, every=7 + b) for b in range(B)])
+    max_len = wl.prompt_len + M + 64
+    kv1 = A.anpd_kv_create(m, max_len, 1)
+    kvb = A.anpd_kv_create(m, max_len, B, True)
+    ctxs = [A.anpd_ngram_create(wl.n_min, wl.n_max, max_len, 0, st) for _ in range(B)]
+    try:
+        A.anpd_kv_set_candidates(kv1, 2)
+        A.anpd_kv_set_candidates(kvb, 2)
+        singles = [A.anpd_generate(m, kv1, ctxs[0], prompts[b], M, K) for b in range(B)]
+        outs, stats = A.anpd_generate_batch(m, kvb, ctxs, prompts, M, K)
+        wins = 0
+        for b in range(B):
+            assert outs[b].tolist() == orbit_continuation(pi, prompts[b][-1], M).tolist()
+            assert np.array_equal(outs[b], singles[b][0]), b
+            _, ost, _ = oracle_two(ScriptedOrbitModel(pi, wl.shape.vocab), prompts[b].tolist(), M, K, n_max=wl.n_max, n_min=wl.n_min)
+            for k in ("steps", "drafted", "accepted", "generated", "hist_accepted", "alt_wins"):
+                assert stats[b][k] == singles[b][1][k], (b, k)
+            assert (stats[b]["steps"], stats[b]["drafted"], stats[b]["accepted"], stats[b]["alt_wins"]) == \
+                   (ost.steps, ost.drafted, ost.accepted, ost.alt_wins)
+            wins += stats[b]["alt_wins"]
+        assert wins > 0
+    finally:
+        for c in ctxs:
+            A.anpd_ngram_destroy(c)
+        A.anpd_kv_destroy(kv1)
+        A.anpd_kv_destroy(kvb)
+        A.anpd_model_destroy(m)
+
+
+def test_two_candidate_error_paths(A):
+    shape = ModelShape(1, 128, 2, 2, 64, 192, 160)
+    w = make_weights(shape, 5, False, std=0.02)
+    m = gpu_model(A, shape, w)
+    kv = A.anpd_kv_create(m, 256)
+    kvb = A.anpd_kv_create(m, 256, 2)
+    try:
+        first = A.anpd_prefill(m, kv, [1, 2, 3, 4, 5])
+        for a, b in [([], [1]), ([1], []), ([1, 2, 3, 4], [1, 2, 3, 4]), ([1], [shape.vocab]), ([-1], [1])]:
+            with pytest.raises(Exception):
+                A.anpd_verify_two_candidates(m, kv, first, a, b)
+        assert A.anpd_kv_len(kv) == 5                                 # nothing was committed by the rejected calls
+        with pytest.raises(Exception):
+            A.anpd_verify_two_candidates(m, kvb, 1, [1], [2])        # batch 1 only
+        for bad in (0, 3, -1):
+            with pytest.raises(Exception):
+                A.anpd_kv_set_candidates(kv, bad)
+        chosen, acc, nxt, _ = A.anpd_verify_two_candidates(m, kv, first, [1], [2])
+        assert chosen in (0, 1) and 0 <= acc <= 1 and A.anpd_kv_len(kv) == 6 + acc
+    finally:
+        A.anpd_kv_destroy(kv)
+        A.anpd_kv_destroy(kvb)
+        A.anpd_model_destroy(m)
