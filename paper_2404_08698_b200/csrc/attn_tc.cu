@@ -333,7 +333,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant_
 // Prompt passes (one query head per kv head): causal attention of a tile of 16 consecutive rows of one head over all the
 // pages those rows may see, page after page with a running maximum, so that no per-page partial leaves the SM and no merge
 // kernel follows.  Products, operand layouts and the page buffer's K -> V^T -> next K rotation are those of the kernel
-// above.  Per page: S^T = K . Q^T; the page's maxima raise the running maxima m; P = 2^(S - m) (hi + lo) goes to shared
+// above.  Per page: S^T = K . Q^T; the page's maxima (folded by eight threads per row, through shared memory) raise the
+// running maxima m, kept by one thread per row; P = 2^(S - m) (hi + lo) goes to shared
 // memory; thread t keeps the sum of its own key's weights, rescaled by 2^(m_old - m) like the output accumulator
 // O[q] (thread = output dimension, in registers), to which O^T = V^T . P^T of the page is added.  The weights' sums are
 // reduced across threads once, at the end.  Pages are visited in ascending order: the result depends on the row's own
@@ -354,8 +355,9 @@ attn_prompt_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     __shared__ uint64_t bar_k[PF_SLOTS], bar_v[PF_SLOTS], bar_s[PF_SLOTS], bar_o[PF_SLOTS];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float red_max[PF_SLOTS][4][PFQ];
+    __shared__ float2 row_ms[PF_SLOTS][PFQ];             // per row: the maximum so far, the factor that rescales older sums to it
     __shared__ float red_sum[PF_SLOTS][4][PFQ];
+    static_assert(PFQ * KV_PAGE * sizeof(float) <= PF_B_BYTES && PFQ * 8 == 128, "the scores of a page pass through the P operand's buffer");
 
     pdl_trigger();
     const int slot = threadIdx.x >> 7, t = threadIdx.x & 127, warp = t >> 5, lane = t & 31;
@@ -410,9 +412,10 @@ attn_prompt_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         fence_async_smem();
         slot_bar(slot);
-        float m_run[PFQ], l_thr[PFQ], o_acc[PFQ];
+        float l_thr[PFQ], o_acc[PFQ];
+        float m_own = -CUDART_INF_F;                     // thread 8q: the running maximum of row q
 #pragma unroll
-        for (int q = 0; q < PFQ; ++q) { m_run[q] = -CUDART_INF_F; l_thr[q] = 0.0f; o_acc[q] = 0.0f; }
+        for (int q = 0; q < PFQ; ++q) { l_thr[q] = 0.0f; o_acc[q] = 0.0f; }
         for (int c = 0; c < n_pages && ok; ++c) {
             // ---- S^T = K . Q^T ----
             if (t == 0) {
@@ -441,30 +444,47 @@ attn_prompt_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 #pragma unroll
                 for (int q = 0; q < PFQ; ++q) s[q] = v[q] + v[PFQ + q];
             }
+            // The page's maxima per row: the scores go through shared memory (the P operand's buffer, free until the
+            // weights are written), transposed so that the eight threads 8q..8q+7 fold row q's 128 keys (16 each, then
+            // three shuffles) instead of every thread folding all 16 rows across its warp.  Thread 8q owns row q's
+            // running maximum: it raises it and leaves the new maximum and the rescaling factor of the row's older sums
+            // in shared memory for everybody.  Words of a row are XOR-ed with 8 * (q & 3): no bank conflicts either way.
             const int key = c * KV_PAGE + t;
+            float* sc = (float*)Ps;
 #pragma unroll
             for (int q = 0; q < PFQ; ++q) {
                 if (key > pos_lo + q) s[q] = -CUDART_INF_F;
-                float mx = s[q];
-                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                if (lane == 0) red_max[slot][warp][q] = mx;
+                sc[q * KV_PAGE + (t ^ ((q & 3) * 8))] = s[q];
             }
             tc_fence_before();
+            slot_bar(slot);
+            {
+                const int q = t >> 3, j = t & 7;
+                float mx = -CUDART_INF_F;
+#pragma unroll
+                for (int i = 0; i < KV_PAGE / 8; ++i) mx = fmaxf(mx, sc[q * KV_PAGE + ((j + 8 * i) ^ ((q & 3) * 8))]);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                if (j == 0) {
+                    const float m_new = fmaxf(m_own, mx);
+                    const bool none = (m_new == -CUDART_INF_F);
+                    row_ms[slot][q] = make_float2(m_new, (none || m_own == -CUDART_INF_F) ? 0.0f : exp2f(m_own - m_new));
+                    m_own = m_new;
+                }
+            }
             slot_bar(slot);
             float scale[PFQ];
 #pragma unroll
             for (int q = 0; q < PFQ; ++q) {
-                const float mp = fmaxf(fmaxf(red_max[slot][0][q], red_max[slot][1][q]), fmaxf(red_max[slot][2][q], red_max[slot][3][q]));
-                const float m_new = fmaxf(m_run[q], mp);
-                const bool none = (m_new == -CUDART_INF_F);
-                scale[q] = (none || m_run[q] == -CUDART_INF_F) ? 0.0f : exp2f(m_run[q] - m_new);
-                const float pw = none ? 0.0f : exp2f(s[q] - m_new);
+                const float2 ms = row_ms[slot][q];
+                scale[q] = ms.y;
+                const float pw = (ms.x == -CUDART_INF_F) ? 0.0f : exp2f(s[q] - ms.x);
                 const bf16 hh = __float2bfloat16_rn(pw);
                 const bf16 ll = __float2bfloat16_rn(pw - __bfloat162float(hh));
                 *(bf16*)(Ps + b_operand_offset<PFN>(q, t)) = hh;
                 *(bf16*)(Ps + b_operand_offset<PFN>(PFQ + q, t)) = ll;
                 l_thr[q] = fmaf(l_thr[q], scale[q], pw);
-                m_run[q] = m_new;
             }
             fence_async_smem();
             slot_bar(slot);
