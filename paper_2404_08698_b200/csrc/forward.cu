@@ -163,12 +163,20 @@ __global__ void __launch_bounds__(NORM_THREADS) embed_img_kernel(const bf16* __r
 __global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restrict__ x, const float* __restrict__ part,
                                                                   const int* __restrict__ seg_count, size_t split_stride, int ld_part,
                                                                   const float* __restrict__ gain, float eps, int d,
-                                                                  bf16* __restrict__ h_hi, bf16* __restrict__ h_lo) {
+                                                                  bf16* __restrict__ h_hi, bf16* __restrict__ h_lo, int ns_max) {
+    // ns_max: the most partial sums any tile of this projection has.  The loads cover that many slabs whatever the tile's own
+    // count (slabs beyond it hold older sums: read, never added), so they do not wait for the count to arrive.
     pdl_trigger();
-    pdl_wait();
     __shared__ float red[32];
     const int row = blockIdx.x, chunks = d >> 2;
-    float4 v[NORM_MAX_CHUNKS];
+    float4 v[NORM_MAX_CHUNKS], gn[NORM_MAX_CHUNKS];
+    // the norm's gain is a weight: nothing of this step writes it, so it is fetched before the dependency wait
+#pragma unroll
+    for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
+        const int c = threadIdx.x + u * NORM_THREADS;
+        gn[u] = (c < chunks) ? *(const float4*)(gain + 4 * c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    pdl_wait();
     float ss = 0.0f;
 #pragma unroll
     for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
@@ -178,11 +186,11 @@ __global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restr
             const int ns = seg_count[(4 * c) >> 7];
             const float* pr = part + (size_t)row * ld_part + 4 * c;
             float4 acc = *(const float4*)(x + (size_t)row * d + 4 * c);
-            for (int s0 = 0; s0 < ns; s0 += 8) {
+            for (int s0 = 0; s0 < ns_max; s0 += 8) {
                 float4 p[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    p[k] = (s0 + k < ns) ? *(const float4*)(pr + (size_t)(s0 + k) * split_stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    p[k] = (s0 + k < ns_max) ? *(const float4*)(pr + (size_t)(s0 + k) * split_stride) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     if (s0 + k < ns) { acc.x += p[k].x; acc.y += p[k].y; acc.z += p[k].z; acc.w += p[k].w; }
@@ -197,7 +205,7 @@ __global__ void __launch_bounds__(NORM_THREADS) resid_norm_kernel(float* __restr
     for (int u = 0; u < NORM_MAX_CHUNKS; ++u) {
         const int c = threadIdx.x + u * NORM_THREADS;
         if (c < chunks) {
-            const float4 g = *(const float4*)(gain + 4 * c);
+            const float4 g = gn[u];
             store_split4(make_float4(v[u].x * rstd * g.x, v[u].y * rstd * g.y, v[u].z * rstd * g.z, v[u].w * rstd * g.w),
                          h_hi + (size_t)row * d + 4 * c, h_lo + (size_t)row * d + 4 * c);
         }
@@ -212,7 +220,7 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
                                        const int* __restrict__ row_ok, const float* __restrict__ rope_cos,
                                        const float* __restrict__ rope_sin, const int* __restrict__ page_table,
                                        int pages_per_seq, int Hq, int Hkv, int hd, float q_scale, bf16* __restrict__ q_hi,
-                                       bf16* __restrict__ q_lo, bf16* __restrict__ kpool_l, bf16* __restrict__ vpool_l) {
+                                       bf16* __restrict__ q_lo, bf16* __restrict__ kpool_l, bf16* __restrict__ vpool_l, int ns_max) {
     pdl_trigger();
     pdl_wait();
     // a block covers blockDim.x / (hd / 2) consecutive heads of one row
@@ -220,9 +228,18 @@ __global__ void qkv_rope_append_kernel(const float* __restrict__ part, const int
     if (head >= Hq + 2 * Hkv) return;
     const float* pr = part + (size_t)row * ld_part + (size_t)head * hd;
     float a = 0.0f, b = 0.0f;
+    // up to four slabs are requested before the tile's own count is known (ns_max: the projection's largest count)
+    float pa[4], pb[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        pa[s] = (s < ns_max) ? pr[s * split_stride + i] : 0.0f;
+        pb[s] = (s < ns_max) ? pr[s * split_stride + i + half] : 0.0f;
+    }
     const int ns = seg_count[(head * hd + i) >> 7];      // a head never straddles a 128-column tile
-    for (int s = 0; s < ns; ++s) { a += pr[s * split_stride + i]; b += pr[s * split_stride + i + half]; }
     const int pos = row_pos[row];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) if (s < ns) { a += pa[s]; b += pb[s]; }
+    for (int s = 4; s < ns; ++s) { a += pr[s * split_stride + i]; b += pr[s * split_stride + i + half]; }
     if (head < Hq + Hkv) {
         const float c = rope_cos[(size_t)pos * half + i], sn = rope_sin[(size_t)pos * half + i];
         const float ra = a * c - b * sn, rb = b * c + a * sn;
@@ -702,16 +719,25 @@ __global__ void __launch_bounds__(32 * COMBINE_SLICES) attn_combine_wide_kernel(
 // SwiGLU epilogue of the gate/up projection
 // ---------------------------------------------------------------------------------------------
 __global__ void swiglu_kernel(const float* __restrict__ part, const int* __restrict__ seg_count, size_t split_stride, int ld_part, int F,
-                              bf16* __restrict__ act_hi, bf16* __restrict__ act_lo) {
+                              bf16* __restrict__ act_hi, bf16* __restrict__ act_lo, int ns_max) {
     pdl_trigger();
     pdl_wait();
     const int row = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= F) return;
     const float* pr = part + (size_t)row * ld_part;
     float gte = 0.0f, up = 0.0f;
+    // up to four slabs are requested before the tile's own count is known (ns_max: the projection's largest count)
+    float pg[4], pu[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        pg[s] = (s < ns_max) ? pr[s * split_stride + j] : 0.0f;
+        pu[s] = (s < ns_max) ? pr[s * split_stride + F + j] : 0.0f;
+    }
     const int ng = seg_count[j >> 7], nu = seg_count[(F + j) >> 7];
-    for (int s = 0; s < ng; ++s) gte += pr[s * split_stride + j];
-    for (int s = 0; s < nu; ++s) up += pr[s * split_stride + F + j];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) { if (s < ng) gte += pg[s]; if (s < nu) up += pu[s]; }
+    for (int s = 4; s < ng; ++s) gte += pr[s * split_stride + j];
+    for (int s = 4; s < nu; ++s) up += pr[s * split_stride + F + j];
     const float v = gte / (1.0f + expf(-gte)) * up;
     bf16 hi, lo;
     split_bf16(v, hi, lo);
@@ -973,7 +999,9 @@ __global__ void move_rows_kernel(bf16* __restrict__ h_hi, bf16* __restrict__ h_l
 }
 
 // One projection of the forward.  Returns the per-tile segment counts its consumer must use.
-anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int rows, const int** seg_count_out) {
+anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int rows, const int** seg_count_out, int* seg_max_out = nullptr) {
+    int seg_max_dummy;
+    if (!seg_max_out) seg_max_out = &seg_max_dummy;
     Workspace& ws = kv->ws;
     const GemmPlan& plan = m->plan[kind];
     const int mode = (rows == kv->batch * ANPD_ROWS) ? 0 : 1;
@@ -985,6 +1013,7 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
     if (kind == GK_DOWN) { a_hi = ws.act_hi; a_lo = ws.act_lo; maps = ws.map_act[mode]; }
     if (m->plain_gemm) {
         *seg_count_out = m->d_ones;
+        *seg_max_out = 1;
         return gemm_plain_enqueue(plan, W, a_hi, a_lo, rows, ws.part, ws.n_max_out, m->stream, &m->prof);
     }
     if (mode == 1) {                                   // a prompt pass: complete sums, one per output
@@ -1002,12 +1031,14 @@ anpd_status gemm_enqueue(anpd_model* m, anpd_kv* kv, int kind, int layer, int ro
         } else {
             *seg_count_out = m->d_const_segs[sched.ksplit];
         }
+        *seg_max_out = std::max(sched.ksplit, sched.tail_split);
         return gemm_pf_enqueue(plan, W, maps[0], maps[1], rows, ws.part, ws.n_max_out, (size_t)ws.r_max * ws.n_max_out, sched, m->num_sms,
                                ws.gemm_err, m->stream, &m->prof);
     }
     ANPD_TRY(gemm_tc_enqueue(plan, W, maps[0], maps[1], rows, ws.nb[mode], ws.part, (size_t)kv->batch * ANPD_ROWS * ws.n_max_out,
                              ws.n_max_out, ws.gemm_err, m->stream, &m->prof));
     *seg_count_out = plan.d_seg_count;
+    *seg_max_out = plan.max_segs;
     return ANPD_OK;
 }
 
@@ -1154,6 +1185,7 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     const size_t sstride = (rows == kv->batch * ANPD_ROWS) ? (size_t)kv->batch * ANPD_ROWS * ws.n_max_out : (size_t)ws.r_max * ws.n_max_out;
     const size_t layer_elems = (size_t)kv->total_pages * c.n_kv_heads * KV_PAGE * hd;
     const int* segs = nullptr;
+    int seg_max = 1;                                   // the most partial sums a tile of the last projection has
 
     LAUNCH(pf, st, KC_OTHER, 0, (launch_k(embed_norm_kernel, rows, NORM_THREADS, 0, st, m->embed, ws.row_tok, m->layers[0].attn_norm, c.rms_eps, d,
                                                                       ws.x, ws.h_hi, ws.h_lo)));
@@ -1161,7 +1193,7 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
     const int rope_hpb = many_rows ? 256 / (hd / 2) : 1;            // heads per block of the rotary kernel
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& w = m->layers[l];
-        ANPD_TRY(gemm_enqueue(m, kv, GK_QKV, l, rows, &segs));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_QKV, l, rows, &segs, &seg_max));
         if (rows != kv->batch * ANPD_ROWS) {            // a prompt pass
             const dim3 grid((rows + ROPE_TILE_ROWS - 1) / ROPE_TILE_ROWS, c.n_q_heads + 2 * c.n_kv_heads);
             const float qs = 1.4426950408889634f / sqrtf((float)hd);
@@ -1178,25 +1210,25 @@ anpd_status forward_enqueue(anpd_model* m, anpd_kv* kv, int rows, int max_pos, b
                (launch_k(qkv_rope_append_kernel, dim3(rows, (c.n_q_heads + 2 * c.n_kv_heads + rope_hpb - 1) / rope_hpb), rope_hpb * (hd / 2), 0, st, 
                    ws.part, segs, sstride, ws.n_max_out, ws.row_pos, ws.row_slot, ws.row_seq, ws.row_ok, kv->rope_cos, kv->rope_sin,
                    kv->page_table, kv->pages_per_seq, c.n_q_heads, c.n_kv_heads, hd, 1.4426950408889634f / sqrtf((float)hd), ws.q_hi,
-                   ws.q_lo, kv->kpool + l * layer_elems, kv->vpool + l * layer_elems)));
+                   ws.q_lo, kv->kpool + l * layer_elems, kv->vpool + l * layer_elems, seg_max)));
         if (hd == 128) ANPD_TRY(attn_enqueue<128>(m, kv, l, rows, max_pos, nullptr, two_candidates));
         else ANPD_TRY(attn_enqueue<64>(m, kv, l, rows, max_pos, nullptr, two_candidates));
-        ANPD_TRY(gemm_enqueue(m, kv, GK_O, l, rows, &segs));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_O, l, rows, &segs, &seg_max));
         LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(resid_norm_kernel, rows, NORM_THREADS, 0, st, ws.x, ws.part, segs, sstride, ws.n_max_out, w.ffn_norm, c.rms_eps, d,
-                                                       ws.h_hi, ws.h_lo)));
-        ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs));
+                                                       ws.h_hi, ws.h_lo, seg_max)));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_GU, l, rows, &segs, &seg_max));
         if (many_rows) LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(swiglu_wide_kernel, dim3((F / 4 + 511) / 512, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
                          ws.act_lo)));
         else LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(swiglu_kernel, dim3((F + 255) / 256, rows), 256, 0, st, ws.part, segs, sstride, ws.n_max_out, F, ws.act_hi,
-                                                                          ws.act_lo)));
-        ANPD_TRY(gemm_enqueue(m, kv, GK_DOWN, l, rows, &segs));
+                                                                          ws.act_lo, seg_max)));
+        ANPD_TRY(gemm_enqueue(m, kv, GK_DOWN, l, rows, &segs, &seg_max));
         const float* next_gain = (l + 1 < c.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
         LAUNCH(pf, st, KC_OTHER, 0,
                (launch_k(resid_norm_kernel, rows, NORM_THREADS, 0, st, ws.x, ws.part, segs, sstride, ws.n_max_out, next_gain, c.rms_eps, d,
-                                                       ws.h_hi, ws.h_lo)));
+                                                       ws.h_hi, ws.h_lo, seg_max)));
     }
     if (!head) { CUDA_TRY(cudaGetLastError()); return ANPD_OK; }
     int head_rows = rows;
