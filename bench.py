@@ -442,6 +442,34 @@ def structured_acceptance(args, A, stream, names) -> list:
             "ms_per_step_anpd": step_a, "ms_per_step_greedy": step_g, "ms_prefill": st_a["ms_prefill"],
             "anpd_equals_greedy": bool(np.array_equal(out_a, out_g)), "equals_closed_form": bool(np.array_equal(out_a, want)),
         })
+    # One candidate per step against two (the paper's outlook; anpd_kv_set_candidates) on a prompt whose long n-gram contexts
+    # mislead while the shortest is right (workloads.orbit_fork_prompt): the case the second candidate exists for.
+    from workloads import orbit_fork_prompt
+    wl = wl0
+    pi = orbit_permutation(wl.orbit_S, wl.weight_seed)
+    prompt = orbit_fork_prompt(pi, wl.prompt_len, wl.prompt_seed)
+    want = orbit_continuation(pi, prompt[-1], wl.max_new)
+    prompt_dev = torch.from_numpy(prompt).cuda()
+    two = {}
+    for label, cands, K in (("one_candidate", 1, 4), ("two_candidates", 2, max(wl.K, 4))):
+        A.anpd_kv_set_candidates(kv, cands)
+        for _ in range(2):
+            A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            st = A.anpd_generate_dev(model, kv, ctx, prompt_dev, wl.max_new, K, out_dev)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        t = e0.elapsed_time(e1) / 1e3 / args.steps
+        two[label] = {"tokens_per_s": wl.max_new / t, "steps": st["steps"], "drafted": st["drafted"], "accepted": st["accepted"],
+                      "steps_won_by_second_candidate": st["alt_wins"], "ms_per_step": st["ms_decode"] / st["steps"],
+                      "equals_closed_form": bool(np.array_equal(out_dev.cpu().numpy(), want))}
+    A.anpd_kv_set_candidates(kv, 1)
+    rows.append({"workload": f"{names[0]} shape and model, forked prompt of {wl.prompt_len} tokens (long contexts mislead, the one-token context is right), "
+                             f"{wl.max_new} new tokens, N={wl.n_max}: one candidate (K=4) against two (4+3) per step", **two,
+                 "speedup_two_over_one": two["two_candidates"]["tokens_per_s"] / two["one_candidate"]["tokens_per_s"]})
     A.anpd_ngram_destroy(ctx)
     A.anpd_kv_destroy(kv)
     A.anpd_model_destroy(model)
