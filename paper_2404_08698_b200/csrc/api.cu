@@ -451,11 +451,14 @@ anpd_status anpd_kv_create(const anpd_model* cm, int max_len, int batch, int shu
 
     // TMA views of the K and V pools for the tensor-core attention: every page of every layer and kv head is 128 rows of hd
     kv->attn_tc = (c.head_dim == 128) && std::getenv("ANPD_ATTN_MMA_SYNC") == nullptr;
+    kv->attn_pf = std::getenv("ANPD_ATTN_PROMPT_TILE16") == nullptr;
     if (kv->attn_tc) {
         const long long pool_rows = (long long)c.n_layers * kv->total_pages * c.n_kv_heads * KV_PAGE;
         anpd_status rc = pool_rows < (1ll << 31) ? ANPD_OK : ANPD_ERR_CAPACITY;
         if (rc == ANPD_OK) rc = make_tmap_bf16(&kv->map_k, kv->kpool, (int)pool_rows, c.head_dim, KV_PAGE, true);
         if (rc == ANPD_OK) rc = make_tmap_bf16(&kv->map_v, kv->vpool, (int)pool_rows, c.head_dim, KV_PAGE, true);
+        if (rc == ANPD_OK) rc = make_tmap_bf16(&ws.map_q[0], ws.q_hi, ws.r_max, m->dq, 128, false);
+        if (rc == ANPD_OK) rc = make_tmap_bf16(&ws.map_q[1], ws.q_lo, ws.r_max, m->dq, 128, false);
         if (rc != ANPD_OK) { cudaFreeHost(kv->h_seq); cudaFree(kv->slab); delete kv; return rc; }
     }
 

@@ -1055,7 +1055,7 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
         CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
     if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && c.n_q_heads == c.n_kv_heads)
-        return attn_prompt_enqueue(m, kv, layer, rows);          // a prompt pass: pages are folded in the kernel, nothing to merge
+        return kv->attn_pf ? attn_pf_enqueue(m, kv, layer, rows) : attn_prompt_enqueue(m, kv, layer, rows);   // a prompt pass: pages are folded in the kernel, nothing to merge
     if (HD == 128 && kv->attn_tc) {
         ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos, tree));
     } else {

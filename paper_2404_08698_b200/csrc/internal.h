@@ -313,6 +313,7 @@ struct Workspace {
     int* gemm_err;                    // device flag set by a GEMM kernel that gave up waiting
     // TMA views of the activation buffers: [0] decode (batch*8 rows), [1] prompt passes (prefill_rows rows, boxes of 128 rows)
     CUtensorMap map_h[2][2], map_ao[2][2], map_act[2][2];     // [mode][hi/lo]
+    CUtensorMap map_q[2];             // the queries of a prompt pass (hi, lo) through boxes of 64 columns x 128 rows (head dimension 128)
     int nb[2];                        // MMA N per mode (rows padded to a multiple of 16)
 };
 
@@ -362,6 +363,7 @@ struct anpd_kv {
     __nv_bfloat16 *kpool, *vpool;     // per layer and page: K [Hkv][KV_PAGE][hd]; V transposed [Hkv][hd][KV_PAGE]
     CUtensorMap map_k, map_v;         // TMA views of the two pools as [all page rows][hd] matrices (head dimension 128 only)
     bool attn_tc;                     // attention on tcgen05 (head dimension 128); otherwise the mma.sync kernel
+    bool attn_pf;                     // prompt passes: the 128-row kernel (attn_pf.cu); otherwise the 16-row kernel of attn_tc.cu
     int* page_table;                  // device [batch][pages_per_seq]
     float *rope_cos, *rope_sin;       // [max_len][hd/2]
     SeqState* seq;                    // device [batch]
@@ -422,6 +424,8 @@ anpd_status accept_enqueue(anpd_model* m, anpd_kv* kv, int mode, const NgramDev*
 // attn_tc.cu: per-page attention partials for head dimension 128 (same outputs as the mma.sync kernel in forward.cu)
 // tree: the rows carry cache slots and hidden slot ranges of their own (two-candidate steps)
 anpd_status attn_tc_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int max_pos, bool tree = false);
+// attn_pf.cu: attention of a prompt pass with 128 query rows per CTA (head dimension 128, one query head per kv head)
+anpd_status attn_pf_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows);
 // attention of a prompt pass (one query head per kv head), written straight to the O projection's input
 anpd_status attn_prompt_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows);
 

@@ -339,3 +339,44 @@ def test_prompt_longer_than_one_pass(A, shape, plen):
     err = float((torch.from_numpy(got).double() - want).abs().max())
     print(f"{plen} tokens, hd {shape.head_dim}: max-abs {err:.2e}")
     assert err <= 5e-3, err
+
+
+@pytest.mark.parametrize("std", [0.05, 0.4])
+def test_prompt_attention_with_128_row_tiles(A, monkeypatch, std):
+    """The prompt-pass attention with the query rows on the tensor-memory lanes (head dimension 128, one query head per kv
+    head): prompts that end inside a row tile, on a page boundary and several tiles in, against the oracle and against the
+    16-rows-per-slot kernel it replaces.  The larger weight scale spreads the scores over many powers of two, so that the
+    lazily moved reference maximum has to move (and the output accumulator be rescaled) inside a prompt."""
+    shape = ModelShape(2, 256, 2, 2, 128, 320, 200)
+    w = make_weights(shape, 17, False, std=std, norm_gain_jitter=0.1)
+    dec = Decoder(shape, as_bf16_values(w), torch.float64, kv_dtype=torch.bfloat16)
+    draft = [int(t) for t in markov_prompt(7, shape.vocab, 2, 5)]
+    for plen in (5, 127, 128, 129, 300, 1000):
+        prompt = markov_prompt(plen, shape.vocab, 2, 100 + plen).tolist()
+        got = {}
+        for old in (False, True):
+            if old:
+                monkeypatch.setenv("ANPD_ATTN_PROMPT_TILE16", "1")
+            else:
+                monkeypatch.delenv("ANPD_ATTN_PROMPT_TILE16", raising=False)
+            m = gpu_model(A, shape, w)
+            kv = A.anpd_kv_create(m, plen + 64, 1, True)
+            try:
+                first = A.anpd_prefill(m, kv, prompt)
+                got[old] = (first, A.anpd_verify_logits(m, kv, first, draft, shape.vocab))
+            finally:
+                A.anpd_kv_destroy(kv)
+                A.anpd_model_destroy(m)
+        monkeypatch.delenv("ANPD_ATTN_PROMPT_TILE16", raising=False)
+        cache = dec.new_cache()
+        lp = dec.forward(prompt, cache)
+        first = got[False][0]
+        if top2_margin(lp[-1]) > 5e-2 * max(1.0, float(lp[-1].abs().max())):
+            assert first == argmax_lowest(lp[-1])
+        want = dec.forward([first] + draft, cache)
+        scale = max(1.0, float(want.abs().max()))
+        err = float((torch.from_numpy(got[False][1]).double() - want).abs().max())
+        assert err <= 5e-3 * scale, (plen, err, scale)
+        if got[True][0] == first:                          # the two kernels sum in different orders: equal up to rounding
+            cross = float(np.abs(got[False][1] - got[True][1]).max())
+            assert cross <= 1e-3 * scale, (plen, cross, scale)
