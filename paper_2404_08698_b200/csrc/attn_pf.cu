@@ -1,6 +1,6 @@
-// Causal attention of a prompt pass (Algorithm 1's LLM(prompt)) for head dimension 128 with one query head per kv head,
-// with the query rows on the tensor-memory lanes: a CTA takes 128 consecutive rows of one head through all the pages those
-// rows may see.
+// Causal attention of a prompt pass (Algorithm 1's LLM(prompt)) for head dimension 128, with the query rows on the
+// tensor-memory lanes: a CTA takes 128 consecutive rows of one query head through all the pages (of its kv head) those rows
+// may see.
 //
 //   S  = Q_hi K^T + Q_lo K^T      128 rows x 128 keys of a page, both terms into one accumulator (thread = row)
 //   m' = rowmax S if that exceeds m by more than 2^8, else m;  P = 2^(S - m')  (hi + lo terms, to shared memory as the next
@@ -48,7 +48,7 @@ __device__ __forceinline__ int fa_offset(int row, int k) {
 struct FaArgs {
     const int* page_table; int pages_per_seq;
     const int* row_pos; const int* row_seq;
-    int H, layer_row0, rows, n_row_tiles;
+    int H, Hkv, layer_row0, rows, n_row_tiles;      // query heads, kv heads (H a multiple of Hkv)
     bf16* ao_hi; bf16* ao_lo;
     int* err;
 };
@@ -139,7 +139,7 @@ attn_pf_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_constant
                     const uint32_t slot = li % FA_RING, use = li / FA_RING;
                     ok = mbar_wait(&ring_empty[slot], (use & 1u) ^ 1u, abortp);
                     if (!ok) break;
-                    const int row = g.layer_row0 + (g.page_table[seq * g.pages_per_seq + c] * g.H + h) * KV_PAGE;
+                    const int row = g.layer_row0 + (g.page_table[seq * g.pages_per_seq + c] * g.Hkv + h / (g.H / g.Hkv)) * KV_PAGE;
                     unsigned char* dst = ring + (size_t)slot * FA_OPER;
                     mbar_expect_tx(&ring_full[slot], FA_OPER);
                     tma_load_2d(dst, kk ? &map_k : &map_v, 0, row, &ring_full[slot], pol);
@@ -366,7 +366,7 @@ anpd_status attn_pf_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows) {
     FaArgs g;
     g.page_table = kv->page_table; g.pages_per_seq = kv->pages_per_seq;
     g.row_pos = ws.row_pos; g.row_seq = ws.row_seq;
-    g.H = c.n_q_heads;
+    g.H = c.n_q_heads; g.Hkv = c.n_kv_heads;
     g.layer_row0 = layer * kv->total_pages * c.n_kv_heads * KV_PAGE;
     g.rows = rows;
     g.n_row_tiles = (rows + FA_ROWS - 1) / FA_ROWS;

@@ -1054,8 +1054,9 @@ anpd_status attn_enqueue(anpd_model* m, anpd_kv* kv, int layer, int rows, int ma
     if (first_call_on_device(attr_set)) {
         CUDA_TRY(cudaFuncSetAttribute(attn_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
-    if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && c.n_q_heads == c.n_kv_heads)
-        return kv->attn_pf ? attn_pf_enqueue(m, kv, layer, rows) : attn_prompt_enqueue(m, kv, layer, rows);   // a prompt pass: pages are folded in the kernel, nothing to merge
+    // a prompt pass: pages are folded in the kernel, nothing to merge (the older 16-row kernel knows one query head per kv head only)
+    if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && kv->attn_pf) return attn_pf_enqueue(m, kv, layer, rows);
+    if (HD == 128 && kv->attn_tc && rows != kv->batch * ANPD_ROWS && c.n_q_heads == c.n_kv_heads) return attn_prompt_enqueue(m, kv, layer, rows);
     if (HD == 128 && kv->attn_tc) {
         ANPD_TRY(attn_tc_enqueue(m, kv, layer, rows, max_pos, tree));
     } else {

@@ -341,15 +341,21 @@ def test_prompt_longer_than_one_pass(A, shape, plen):
     assert err <= 5e-3, err
 
 
+@pytest.mark.parametrize("heads", [(2, 2), (4, 2), (4, 1)], ids=lambda h: f"g{h[0] // h[1]}")
 @pytest.mark.parametrize("std", [0.05, 0.4])
-def test_prompt_attention_with_128_row_tiles(A, monkeypatch, std):
-    """The prompt-pass attention with the query rows on the tensor-memory lanes (head dimension 128, one query head per kv
-    head): prompts that end inside a row tile, on a page boundary and several tiles in, against the oracle and against the
-    16-rows-per-slot kernel it replaces.  The larger weight scale spreads the scores over many powers of two, so that the
+def test_prompt_attention_with_128_row_tiles(A, monkeypatch, std, heads):
+    """The prompt-pass attention with the query rows on the tensor-memory lanes (head dimension 128; 1, 2 and 4 query heads
+    per kv head): prompts that end inside a row tile, on a page boundary and several tiles in, against the oracle and against
+    the kernels it replaces (16 rows per slot; page partials + merge where query heads share a kv head).  At the larger
+    weight scale the softmax is close to an argmax and the model amplifies any rounding: there the bar against the oracle
+    is the oracle's own sensitivity to the cache's bf16 rounding (its distance to itself with a full-precision cache), as
+    in the deep-model tests, and the comparison with the replaced kernels (same cache, same roundings elsewhere) is the
+    sharp one.  The larger weight scale spreads the scores over many powers of two, so that the
     lazily moved reference maximum has to move (and the output accumulator be rescaled) inside a prompt."""
-    shape = ModelShape(2, 256, 2, 2, 128, 320, 200)
+    shape = ModelShape(2, 256, heads[0], heads[1], 128, 320, 200)
     w = make_weights(shape, 17, False, std=std, norm_gain_jitter=0.1)
     dec = Decoder(shape, as_bf16_values(w), torch.float64, kv_dtype=torch.bfloat16)
+    dec_plain = Decoder(shape, as_bf16_values(w), torch.float64)
     draft = [int(t) for t in markov_prompt(7, shape.vocab, 2, 5)]
     for plen in (5, 127, 128, 129, 300, 1000):
         prompt = markov_prompt(plen, shape.vocab, 2, 100 + plen).tolist()
@@ -376,7 +382,10 @@ def test_prompt_attention_with_128_row_tiles(A, monkeypatch, std):
         want = dec.forward([first] + draft, cache)
         scale = max(1.0, float(want.abs().max()))
         err = float((torch.from_numpy(got[False][1]).double() - want).abs().max())
-        assert err <= 5e-3 * scale, (plen, err, scale)
+        cp = dec_plain.new_cache()
+        dec_plain.forward(prompt, cp)
+        cache_effect = float((dec_plain.forward([first] + draft, cp) - want).abs().max())
+        assert err <= max(5e-3 * scale, cache_effect), (plen, err, scale, cache_effect)
         if got[True][0] == first:                          # the two kernels sum in different orders: equal up to rounding
             cross = float(np.abs(got[False][1] - got[True][1]).max())
             assert cross <= 1e-3 * scale, (plen, cross, scale)
